@@ -1,0 +1,188 @@
+"""ctypes front end of the CPU oracle (``skipkv_oracle.cpp``).  TEST INFRASTRUCTURE ONLY.
+
+Only the tests, the smoke check and the benchmark's cpu-baseline / reference legs may
+import this package; the CUDA product path never does.  It takes and returns numpy
+arrays (bf16 tensors travel as ``uint16`` bit patterns) and shares no code with the
+CUDA library.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+from typing import Optional
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "skipkv_oracle.cpp")
+_LIB = os.path.join(_HERE, "libskipkv_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with g++ -O2 -fopenmp (no fast-math) if it is stale."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + f".tmp{os.getpid()}"
+        subprocess.run(["g++", "-std=c++17", "-O2", "-fopenmp", "-fPIC", "-shared", "-o", tmp, _SRC],
+                       check=True)
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        _lib = C.CDLL(build())
+        _lib.oracle_select.restype = C.c_int
+        _lib.oracle_compact.restype = C.c_int
+        _lib.oracle_compact_batch.restype = C.c_int
+        _lib.oracle_max_threads.restype = C.c_int
+    return _lib
+
+
+def _p(a: Optional[np.ndarray]):
+    return None if a is None else a.ctypes.data_as(C.c_void_p)
+
+
+def _c(a, dt):
+    a = np.ascontiguousarray(a, dtype=dt)
+    return a
+
+
+def max_threads() -> int:
+    return int(lib().oracle_max_threads())
+
+
+def set_threads(n: int) -> None:
+    lib().oracle_set_threads(C.c_int(n))
+
+
+# ------------------------------------------------------------------ per-slab functions
+def token_importance(K_bits, Q_bits):
+    """K_bits uint16 [N,d]; Q_bits uint16 [n,alpha,d] -> tok_imp float64 [N]."""
+    K_bits = _c(K_bits, np.uint16); Q_bits = _c(Q_bits, np.uint16)
+    N, d = K_bits.shape
+    n, alpha, d2 = Q_bits.shape
+    assert d == d2
+    out = np.zeros(N, np.float64)
+    lib().oracle_token_importance(_p(K_bits), _p(Q_bits), N, n, alpha, d, _p(out))
+    return out
+
+
+def pool(K_bits, sent_off, tok_imp, eps=1e-6):
+    K_bits = _c(K_bits, np.uint16); sent_off = _c(sent_off, np.int32); tok_imp = _c(tok_imp, np.float64)
+    S = len(sent_off) - 1
+    d = K_bits.shape[1]
+    imp = np.zeros(S, np.float64); vbar = np.zeros((S, d), np.float64)
+    lib().oracle_pool(_p(K_bits), d, _p(sent_off), S, _p(tok_imp), C.c_double(eps), _p(imp), _p(vbar))
+    return imp, vbar
+
+
+def gram_terms(vbar, tau):
+    vbar = _c(vbar, np.float64)
+    S, d = vbar.shape
+    G = np.zeros((S, S), np.float64); red = np.zeros(S, np.float64); lam = np.zeros(S, np.float64)
+    lib().oracle_gram_terms(_p(vbar), S, d, C.c_double(tau), _p(G), _p(red), _p(lam))
+    return G, red, lam
+
+
+def final_score(imp, red, lam, sigma):
+    imp = _c(imp, np.float64); red = _c(red, np.float64); lam = _c(lam, np.float64)
+    out = np.zeros(len(imp), np.float32)
+    lib().oracle_final_score(_p(imp), _p(red), _p(lam), len(imp), C.c_double(sigma), _p(out))
+    return out
+
+
+def select(score, sent_off, budget, protect_tail):
+    score = _c(score, np.float32); sent_off = _c(sent_off, np.int32)
+    S = len(sent_off) - 1
+    keep = np.zeros(S, np.uint8); kept = np.zeros(max(S, 1), np.int32); nl = np.zeros(1, np.int32)
+    nk = lib().oracle_select(_p(score), _p(sent_off), S, int(budget), int(protect_tail), _p(keep), _p(kept), _p(nl))
+    return keep, kept[:nk].copy(), int(nl[0])
+
+
+def compact(K_bits, V_bits, keep, sent_off, sent_id):
+    K_bits = _c(K_bits, np.uint16); V_bits = _c(V_bits, np.uint16)
+    keep = _c(keep, np.uint8); sent_off = _c(sent_off, np.int32); sent_id = _c(sent_id, np.int32)
+    S = len(sent_off) - 1
+    N, d = K_bits.shape
+    Ko = np.zeros_like(K_bits); Vo = np.zeros_like(V_bits)
+    im = np.zeros(max(N, 1), np.int32); nso = np.zeros(S + 1, np.int32); nsid = np.zeros(max(S, 1), np.int32)
+    nl = np.zeros(1, np.int32)
+    ns = lib().oracle_compact(_p(K_bits), _p(V_bits), d, _p(keep), _p(sent_off), _p(sent_id), S, _p(Ko), _p(Vo),
+                              _p(im), _p(nso), _p(nsid), _p(nl))
+    if ns < 0:
+        raise AssertionError("literal range remap disagrees with the prefix-sum form")
+    n = int(nl[0])
+    return Ko[:n], Vo[:n], im[:n], nso[:ns + 1], nsid[:ns]
+
+
+def decode_attn(q_bits, K_bits, V_bits, length):
+    q_bits = _c(q_bits, np.uint16); K_bits = _c(K_bits, np.uint16); V_bits = _c(V_bits, np.uint16)
+    n, d = q_bits.shape
+    out = np.zeros((n, d), np.uint16); o64 = np.zeros((n, d), np.float64)
+    lib().oracle_decode_attn(_p(q_bits), _p(K_bits), _p(V_bits), int(length), n, d, _p(out), _p(o64))
+    return out, o64
+
+
+def steer(hidden_bits, v_bits, alpha, flag):
+    h = _c(hidden_bits, np.uint16).copy(); v = _c(v_bits, np.uint16)
+    alpha = _c(alpha, np.float32); flag = _c(flag, np.uint8)
+    b, dm = h.shape
+    lib().oracle_steer(b, dm, _p(h), _p(v), _p(alpha), _p(flag))
+    return h
+
+
+# ------------------------------------------------------------------ batch drivers
+def score_batch(shape, K_bits, qwin_bits, kv_len, sent_off, n_sent, sigma, tau, eps, want_tok_imp=False):
+    """shape: dict(batch,Hq,Hk,d,alpha,max_sent,slab_off,cap).  Returns dict of arrays."""
+    b, Hq, Hk, d, alpha, ms = (shape[k] for k in ("batch", "Hq", "Hk", "d", "alpha", "max_sent"))
+    slab_off = _c(shape["slab_off"], np.int64); cap = _c(shape["cap"], np.int32)
+    K_bits = _c(K_bits, np.uint16); qwin_bits = _c(qwin_bits, np.uint16)
+    kv_len = _c(kv_len, np.int32); sent_off = _c(sent_off, np.int32); n_sent = _c(n_sent, np.int32)
+    ti = np.zeros(K_bits.shape[0], np.float64) if want_tok_imp else None
+    imp = np.zeros((b, Hk, ms), np.float64); red = np.zeros_like(imp); lam = np.zeros_like(imp)
+    sc = np.zeros((b, Hk, ms), np.float32)
+    lib().oracle_score_batch(b, Hq, Hk, d, alpha, ms, _p(slab_off), _p(cap), _p(K_bits), _p(qwin_bits),
+                             _p(kv_len), _p(sent_off), _p(n_sent), C.c_double(sigma), C.c_double(tau),
+                             C.c_double(eps), _p(ti), _p(imp), _p(red), _p(lam), _p(sc))
+    return dict(tok_imp=ti, imp=imp, red=red, lam=lam, score=sc)
+
+
+def select_batch(score, sent_off, n_sent, budget, protect_tail):
+    score = _c(score, np.float32); sent_off = _c(sent_off, np.int32); n_sent = _c(n_sent, np.int32)
+    ms = score.shape[-1]
+    ns = int(np.prod(score.shape[:-1]))
+    keep = np.zeros(score.shape, np.uint8); kept = np.full(score.shape, -1, np.int32)
+    nk = np.zeros(score.shape[:-1], np.int32); nl = np.zeros(score.shape[:-1], np.int32)
+    lib().oracle_select_batch(ns, ms, _p(score), _p(sent_off), _p(n_sent), int(budget), int(protect_tail),
+                              _p(keep), _p(kept), _p(nk), _p(nl))
+    return dict(keep=keep, kept_idx=kept, n_kept=nk, new_len=nl)
+
+
+def compact_batch(shape, K_bits, V_bits, keep, sent_off, sent_id, n_sent, kv_len, want_index_map=True):
+    """Returns new copies: K, V, sent_off, sent_id, n_sent, kv_len, index_map."""
+    b, Hk, d, ms = (shape[k] for k in ("batch", "Hk", "d", "max_sent"))
+    slab_off = _c(shape["slab_off"], np.int64); cap = _c(shape["cap"], np.int32)
+    K = _c(K_bits, np.uint16).copy(); V = _c(V_bits, np.uint16).copy()
+    keep = _c(keep, np.uint8)
+    so = _c(sent_off, np.int32).copy(); sid = _c(sent_id, np.int32).copy()
+    ns = _c(n_sent, np.int32).copy(); kl = _c(kv_len, np.int32).copy()
+    im = np.full(K.shape[0], -1, np.int32) if want_index_map else None
+    rc = lib().oracle_compact_batch(b, Hk, d, ms, _p(slab_off), _p(cap), _p(K), _p(V), _p(keep), _p(so), _p(sid),
+                                    _p(ns), _p(kl), _p(im))
+    if rc != 0:
+        raise AssertionError("literal range remap disagrees with the prefix-sum form")
+    return dict(K=K, V=V, sent_off=so, sent_id=sid, n_sent=ns, kv_len=kl, index_map=im)
+
+
+def decode_attn_batch(shape, q_bits, K_bits, V_bits, kv_len):
+    b, Hq, Hk, d = (shape[k] for k in ("batch", "Hq", "Hk", "d"))
+    slab_off = _c(shape["slab_off"], np.int64); cap = _c(shape["cap"], np.int32)
+    q_bits = _c(q_bits, np.uint16); K_bits = _c(K_bits, np.uint16); V_bits = _c(V_bits, np.uint16)
+    kv_len = _c(kv_len, np.int32)
+    out = np.zeros((b, Hq, d), np.uint16); o64 = np.zeros((b, Hq, d), np.float64)
+    lib().oracle_decode_attn_batch(b, Hq, Hk, d, _p(slab_off), _p(cap), _p(q_bits), _p(K_bits), _p(V_bits),
+                                   _p(kv_len), _p(out), _p(o64))
+    return out, o64
