@@ -1,0 +1,183 @@
+/*
+ * skipkv.h -- C ABI of the B200 (sm_100a) hot path of SkipKV sentence-level KV eviction.
+ *
+ * Five operations, one per step of the path (paper: Section 4.1 "Skipping KV Storage with
+ * Sentence-level Scoring", Section 4.2 "Skipping KV Generation with Adaptive Steering",
+ * Algorithm 1 "Skipping KV Cache Storage"):
+ *
+ *   skipkv_score        sentence scores per (sequence, KV head)
+ *   skipkv_select       which sentences survive under the KV budget
+ *   skipkv_compact      in-place packing of the surviving K/V rows + range-table update
+ *   skipkv_decode_attn  GQA decode attention over the ragged, compacted cache
+ *   skipkv_steer        steering-vector add on the hidden state
+ *
+ * Conventions
+ *   - Every pointer marked "device" is a CUDA device pointer; "host" is ordinary memory.
+ *   - bf16 tensors are passed as void* (raw 16-bit patterns); head_dim must be 128.
+ *   - Every call only enqueues work on `stream` (a cudaStream_t passed as void*; NULL is the
+ *     default stream).  No call synchronises, allocates device memory or keeps state, except
+ *     skipkv_status, which synchronises the stream to read one word back.
+ *   - The caller owns every buffer.  Scratch memory comes from a caller-provided workspace of
+ *     at least skipkv_workspace_bytes() bytes, 256-byte aligned, prepared once with
+ *     skipkv_workspace_init().  One workspace serves one stream at a time.
+ *   - Return value: 0 on success, a negative SKIPKV_ERR_* otherwise.  Nothing is enqueued
+ *     when an argument check fails.  Device-side problems that cannot be seen at enqueue
+ *     time (a bounded wait that ran out) are recorded in the workspace's status word.
+ *   - No C++ exception crosses this boundary.
+ *
+ * Cache layout ("ragged slabs")
+ *   One K and one V buffer per layer, bf16, rows of head_dim elements (256 bytes).  Sequence
+ *   b owns rows [slab_off[b]*Hk, (slab_off[b]+cap[b])*Hk).  Inside that block KV head h owns
+ *   cap[b] consecutive rows; the first kv_len[b][h] of them are live.  Row of (b, h, t):
+ *   slab_off[b]*Hk + h*cap[b] + t.  There is no padding between sequences.
+ *
+ * Sentence tables (the cache-space range list M^(cs) of Algorithm 1), per (b, h):
+ *   sent_off[b][h][0..max_sent]  token offsets, CSR: sentence i covers [sent_off[i], sent_off[i+1]);
+ *                                sent_off[n_sent] == kv_len[b][h]
+ *   sent_id [b][h][0..max_sent)  generation-space index of each sentence (the mapping Phi)
+ *   n_sent  [b][h]
+ */
+#ifndef SKIPKV_H_
+#define SKIPKV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SKIPKV_OK               0
+#define SKIPKV_ERR_INVALID_ARG (-1)  /* null pointer, negative size, inconsistent shape      */
+#define SKIPKV_ERR_UNSUPPORTED (-2)  /* head_dim != 128, Hq % Hk != 0, group or window too big */
+#define SKIPKV_ERR_WORKSPACE   (-3)  /* workspace null or misaligned                          */
+#define SKIPKV_ERR_CUDA        (-4)  /* a CUDA runtime call failed; see skipkv_last_cuda_error */
+#define SKIPKV_ERR_TIMEOUT     (-5)  /* reported by skipkv_status: a bounded device wait ran out */
+
+/* Bits of the device status word (skipkv_status). */
+#define SKIPKV_STATUS_COMPACT_TIMEOUT 0x1u  /* compaction hand-off wait ran out; rows of that slab are unspecified */
+#define SKIPKV_STATUS_COPY_TIMEOUT    0x2u  /* a bulk copy did not complete within the wait limit */
+#define SKIPKV_STATUS_BAD_TABLE       0x4u  /* a sentence table was inconsistent (offsets beyond cap, n_sent > max_sent) */
+
+typedef struct {
+    int32_t batch;        /* sequences                                                        */
+    int32_t n_q_heads;    /* Hq                                                               */
+    int32_t n_kv_heads;   /* Hk; Hq % Hk == 0, group n = Hq/Hk <= 8                           */
+    int32_t head_dim;     /* must be 128                                                      */
+    int32_t window;       /* observation window alpha (recent queries), n*alpha <= 512        */
+    int32_t d_model;      /* hidden size of the steering add; multiple of 8                   */
+    int32_t max_sent;     /* row stride of the sentence tables; every n_sent <= max_sent      */
+    int32_t max_cap;      /* host-known upper bound of cap[b] (sizes grids and the workspace) */
+    const int64_t* slab_off; /* device [batch], in tokens                                     */
+    const int32_t* cap;      /* device [batch], rows per (sequence, head)                     */
+} skipkv_shape;
+
+typedef struct {
+    float   sigma;        /* importance/redundancy trade-off of the final score (paper: 0.1)  */
+    float   tau;          /* similarity threshold of the redundant set (paper: 0.95..0.99)    */
+    float   eps;          /* added to the norm of a pooled key                                */
+    int32_t budget;       /* KV budget B in tokens per (sequence, head)                       */
+    int32_t protect_tail; /* sentences touching the last protect_tail tokens are always kept  */
+} skipkv_params;
+
+/* Bytes of workspace needed for `shape` (host computation only). */
+int skipkv_workspace_bytes(const skipkv_shape* shape, size_t* bytes);
+
+/* Zero the workspace's counters and status word.  Once per workspace, and again after
+ * skipkv_status reported an error.  ws: device. */
+int skipkv_workspace_init(const skipkv_shape* shape, void* ws, void* stream);
+
+/* Read and clear the device status word.  Synchronises `stream`.  *status_bits (host,
+ * nullable) receives the SKIPKV_STATUS_* bits; returns SKIPKV_ERR_TIMEOUT if a wait ran out. */
+int skipkv_status(void* ws, void* stream, uint32_t* status_bits);
+
+/* Text of the last CUDA error seen by this library on the calling thread (host string). */
+const char* skipkv_last_cuda_error(void);
+
+/*
+ * skipkv_score -- Section 4.1: token importance from the observation window (attention
+ * equation, max over the heads of a group, mean over the window), sentence embeddings by mean
+ * pooling, pairwise sentence similarity (Eq. "PSS"), the redundant set P, the redundancy term
+ * (token-redundancy equation taken over sentences) and the final score (Eq. "I_final").
+ * Per (b, h) slab with N = kv_len[b][h] live rows and S = n_sent[b][h] sentences:
+ *   tok_imp[t]  = (1/alpha) sum_w max_{q in group h} softmax_t(q_win[b][q][w] . K[t] / sqrt(d))
+ *   sent_imp[i] = mean of tok_imp over sentence i
+ *   vbar_i      = mean of K rows of sentence i, divided by (its 2-norm + eps)
+ *   G_ij        = vbar_i . vbar_j
+ *   sent_red[i] = (1/S) sum_{j != i} exp(G_ji) / sum_{k != j} exp(G_jk)
+ *   sent_lam[i] = max_{j > i} G_ij if that is > tau, else 0
+ *   sent_score[i] = sigma*sent_imp[i] - (1-sigma)*sent_red[i] - sent_lam[i]
+ * K: device bf16 (layout above, read only).  q_win: device bf16 [batch][Hq][window][128].
+ * kv_len: device [batch][Hk].  sent_off / n_sent: device tables (read only).
+ * tok_imp: device fp32, one value per cache row with the row indexing of K, nullable
+ * (then it lives in the workspace).  sent_imp, sent_red, sent_lam, sent_score: device fp32
+ * [batch][Hk][max_sent]; entries at i >= n_sent are not written.
+ */
+int skipkv_score(const skipkv_shape* shape, const skipkv_params* params, const void* K,
+                 const void* q_win, const int32_t* kv_len, const int32_t* sent_off,
+                 const int32_t* n_sent, float* tok_imp, float* sent_imp, float* sent_red,
+                 float* sent_lam, float* sent_score, void* ws, void* stream);
+
+/*
+ * skipkv_select -- Section 4.1 (evict in increasing order of the final score until the cache
+ * meets the budget B), at whole-sentence granularity.  Per slab: if kv_len <= budget keep
+ * everything.  Otherwise rank sentences: those touching the last protect_tail tokens first (in
+ * index order), then by (score descending, index ascending, exact fp32 comparison); walk the
+ * ranking summing sentence lengths and keep the longest prefix whose total is <= budget (the
+ * walk stops at the first sentence that does not fit).  Scores must not be NaN.
+ * keep: device u8 [batch][Hk][max_sent] (1 = survives; entries >= n_sent set to 0).
+ * kept_idx: device int32 [batch][Hk][max_sent], ascending sentence indices, nullable.
+ * n_kept, new_len: device int32 [batch][Hk] (new_len = surviving tokens), nullable.
+ */
+int skipkv_select(const skipkv_shape* shape, const skipkv_params* params, const float* sent_score,
+                  const int32_t* sent_off, const int32_t* n_sent, uint8_t* keep, int32_t* kept_idx,
+                  int32_t* n_kept, int32_t* new_len, void* ws, void* stream);
+
+/*
+ * skipkv_compact -- Algorithm 1, eviction and post-eviction update (Eq. "after"): the rows of
+ * the kept sentences move down, in their original order, to rows [0, new_len) of the same slab,
+ * for K and for V, in place.  The range tables are rewritten: sent_off becomes the exclusive
+ * prefix sum of the kept lengths (entries above the new n_sent are set to new_len), sent_id is
+ * filtered (tail set to -1), n_sent and kv_len are updated; sentences with no surviving token
+ * disappear.  index_map (device int32, one entry per cache row, row indexing of K, nullable):
+ * index_map[row of (b,h,k)] = old token index of new token k, for k < new_len.
+ * Rows at and beyond new_len are unspecified afterwards.  Moved rows are bit-identical copies.
+ */
+int skipkv_compact(const skipkv_shape* shape, void* K, void* V, const uint8_t* keep,
+                   int32_t* sent_off, int32_t* sent_id, int32_t* n_sent, int32_t* kv_len,
+                   int32_t* index_map, void* ws, void* stream);
+
+/*
+ * skipkv_decode_attn -- the attention equation of Section 4.1 with one query per head over the
+ * live rows of each slab: out[b][q] = sum_t softmax_t(q[b][q] . K[t] / sqrt(d)) V[t] for
+ * t < kv_len[b][q / n]; fp32 accumulation, bf16 result; kv_len == 0 gives zeros.
+ * q, out: device bf16 [batch][Hq][128].  If hidden is non-null the steering add of
+ * skipkv_steer is performed on it by the same launch (arguments as below).
+ */
+int skipkv_decode_attn(const skipkv_shape* shape, const void* q, const void* K, const void* V,
+                       const int32_t* kv_len, void* out, void* hidden, const void* steer_vec,
+                       const float* alpha, const uint8_t* flag, void* ws, void* stream);
+
+/*
+ * skipkv_steer -- Section 4.2: H <- H + alpha_t * v for the sequences whose current token is a
+ * delimiter.  hidden: device bf16 [batch][d_model], in place.  steer_vec: device bf16
+ * [d_model].  alpha: device fp32 [batch] (alpha_0 + gamma*N_o, computed by the caller).
+ * flag: device u8 [batch], rows with 0 are untouched.  One fp32 fused multiply-add per
+ * element, rounded to nearest even bf16.
+ */
+int skipkv_steer(int32_t batch, int32_t d_model, void* hidden, const void* steer_vec,
+                 const float* alpha, const uint8_t* flag, void* stream);
+
+/*
+ * skipkv_append -- pre-eviction bookkeeping of Algorithm 1 for one decode step: writes the new
+ * K/V row of every (b, h) at position kv_len[b][h] and increments kv_len.  k_new, v_new:
+ * device bf16 [batch][Hk][128].  A slab that is already full (kv_len == cap) is left
+ * unchanged and SKIPKV_STATUS_BAD_TABLE is raised in the status word of ws.
+ */
+int skipkv_append(const skipkv_shape* shape, void* K, void* V, const void* k_new, const void* v_new,
+                  int32_t* kv_len, void* ws, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SKIPKV_H_ */

@@ -1,0 +1,98 @@
+// Workspace management, argument checks and error reporting of the SkipKV C ABI.
+#include <cstdio>
+#include <cstring>
+
+#include "common.cuh"
+
+namespace skipkv {
+
+static thread_local char g_err[256] = "";
+
+int cuda_fail(cudaError_t e) {
+    std::snprintf(g_err, sizeof(g_err), "%s: %s", cudaGetErrorName(e), cudaGetErrorString(e));
+    return SKIPKV_ERR_CUDA;
+}
+
+int num_sms() {
+    static thread_local int cached_dev = -1, cached = 0;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+    if (dev != cached_dev) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+        cached = n;
+        cached_dev = dev;
+    }
+    return cached;
+}
+
+int check_shape(const skipkv_shape* s) {
+    if (!s) return SKIPKV_ERR_INVALID_ARG;
+    if (s->batch <= 0 || s->n_q_heads <= 0 || s->n_kv_heads <= 0 || s->window <= 0 || s->max_sent < 0 ||
+        s->max_cap <= 0 || s->d_model < 0)
+        return SKIPKV_ERR_INVALID_ARG;
+    if (!s->slab_off || !s->cap) return SKIPKV_ERR_INVALID_ARG;
+    if (s->head_dim != kHeadDim) return SKIPKV_ERR_UNSUPPORTED;
+    if (s->n_q_heads % s->n_kv_heads != 0) return SKIPKV_ERR_UNSUPPORTED;
+    const int group = s->n_q_heads / s->n_kv_heads;
+    if (group > kMaxGroup || group * s->window > kMaxQRows) return SKIPKV_ERR_UNSUPPORTED;
+    if (s->d_model % 8 != 0) return SKIPKV_ERR_UNSUPPORTED;
+    if (int64_t(s->batch) * s->n_kv_heads > (1 << 20)) return SKIPKV_ERR_UNSUPPORTED;
+    return SKIPKV_OK;
+}
+
+__global__ void ws_clear_kernel(uint32_t* p, size_t n_words) {
+    for (size_t i = blockIdx.x * size_t(blockDim.x) + threadIdx.x; i < n_words; i += size_t(gridDim.x) * blockDim.x)
+        p[i] = 0u;
+}
+
+}  // namespace skipkv
+
+using namespace skipkv;
+
+extern "C" {
+
+int skipkv_workspace_bytes(const skipkv_shape* shape, size_t* bytes) {
+    if (!bytes) return SKIPKV_ERR_INVALID_ARG;
+    // slab_off / cap are not needed to size the workspace
+    if (!shape) return SKIPKV_ERR_INVALID_ARG;
+    skipkv_shape s = *shape;
+    static const int64_t dummy_off = 0;
+    static const int32_t dummy_cap = 0;
+    if (!s.slab_off) s.slab_off = &dummy_off;
+    if (!s.cap) s.cap = &dummy_cap;
+    if (int rc = check_shape(&s)) return rc;
+    *bytes = make_layout(s).total;
+    return SKIPKV_OK;
+}
+
+int skipkv_workspace_init(const skipkv_shape* shape, void* ws, void* stream) {
+    if (int rc = check_shape(shape)) return rc;
+    if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255)) return SKIPKV_ERR_WORKSPACE;
+    const WsLayout L = make_layout(*shape);
+    // header + every counter region (everything before the decode partials)
+    const size_t words = L.dec_part / 4;
+    ws_clear_kernel<<<64, 256, 0, static_cast<cudaStream_t>(stream)>>>(static_cast<uint32_t*>(ws), words);
+    SKIPKV_CUDA(cudaGetLastError());
+    return SKIPKV_OK;
+}
+
+int skipkv_status(void* ws, void* stream, uint32_t* status_bits) {
+    if (!ws) return SKIPKV_ERR_WORKSPACE;
+    uint32_t bits = 0;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    SKIPKV_CUDA(cudaMemcpyAsync(&bits, ws, sizeof(bits), cudaMemcpyDeviceToHost, st));
+    SKIPKV_CUDA(cudaStreamSynchronize(st));
+    if (bits) {
+        SKIPKV_CUDA(cudaMemsetAsync(ws, 0, sizeof(bits), st));
+        SKIPKV_CUDA(cudaStreamSynchronize(st));
+    }
+    if (status_bits) *status_bits = bits;
+    if (bits & (SKIPKV_STATUS_COMPACT_TIMEOUT | SKIPKV_STATUS_COPY_TIMEOUT)) return SKIPKV_ERR_TIMEOUT;
+    if (bits & SKIPKV_STATUS_BAD_TABLE) return SKIPKV_ERR_INVALID_ARG;
+    return SKIPKV_OK;
+}
+
+const char* skipkv_last_cuda_error(void) { return g_err; }
+
+}  // extern "C"

@@ -1,0 +1,161 @@
+// Shared host/device helpers of the SkipKV CUDA library (sm_100a only).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "skipkv.h"
+
+namespace skipkv {
+
+constexpr int kHeadDim = 128;
+constexpr int kRowBytes = kHeadDim * 2;       // one bf16 K or V row
+constexpr int kMaxGroup = 8;                  // query heads per KV head
+constexpr int kMaxQRows = 512;                // group * window
+
+// ---------------------------------------------------------------------------------------
+// Workspace layout.  All offsets are multiples of 256 bytes from the workspace base.
+// ---------------------------------------------------------------------------------------
+struct Header {                // first 256 bytes of the workspace
+    uint32_t status;           // SKIPKV_STATUS_* bits
+    uint32_t compact_ticket;   // dynamic segment scheduler of the compaction kernel
+    uint32_t pad[62];
+};
+
+struct WsLayout {
+    size_t header;
+    size_t cp_nseg;        // int32  [slabs]              segments per stream
+    size_t cp_loaded;      // uint32 [2*slabs]            segments whose loads are complete
+    size_t cp_nruns;       // int32  [slabs]
+    size_t cp_run_src;     // int32  [slabs][max_sent]    first source token of a run
+    size_t cp_run_dst;     // int32  [slabs][max_sent+1]  first destination token; [nruns] = new_len
+    size_t dec_cnt;        // uint32 [slabs]              partials that arrived (self-resetting)
+    size_t dec_part;       // float  [max_ctas + slabs][group][130]
+    size_t sc_part;        // float2 [slabs][sc_chunks][qrows]  (max, sum) of a chunk of logits
+    size_t sc_lse;         // float  [slabs][qrows]
+    size_t sc_tokimp;      // float  [slabs][max_cap]
+    size_t sc_vbar;        // float  [slabs][max_sent][128]
+    size_t sc_z;           // float  [slabs][max_sent]
+    size_t total;
+    int slabs, group, qrows, sc_chunks, dec_max_ctas;
+};
+
+constexpr int kScoreChunk = 1024;     // tokens per sweep-1 CTA
+constexpr int kDecMaxCtas = 1024;     // upper bound of the decode grid
+
+inline size_t align256(size_t x) { return (x + 255) & ~size_t(255); }
+
+inline WsLayout make_layout(const skipkv_shape& s) {
+    WsLayout L{};
+    L.slabs = s.batch * s.n_kv_heads;
+    L.group = s.n_q_heads / s.n_kv_heads;
+    L.qrows = L.group * s.window;
+    L.sc_chunks = (s.max_cap + kScoreChunk - 1) / kScoreChunk;
+    if (L.sc_chunks < 1) L.sc_chunks = 1;
+    L.dec_max_ctas = kDecMaxCtas;
+    size_t o = 0;
+    auto take = [&](size_t bytes) { size_t r = o; o = align256(o + bytes); return r; };
+    const size_t slabs = L.slabs, ms = s.max_sent > 0 ? s.max_sent : 1;
+    L.header = take(sizeof(Header));
+    L.cp_nseg = take(slabs * 4);
+    L.cp_loaded = take(slabs * 2 * 4);
+    L.cp_nruns = take(slabs * 4);
+    L.cp_run_src = take(slabs * ms * 4);
+    L.cp_run_dst = take(slabs * (ms + 1) * 4);
+    L.dec_cnt = take(slabs * 4);
+    L.dec_part = take((size_t(L.dec_max_ctas) + slabs) * L.group * 130 * 4);
+    L.sc_part = take(slabs * L.sc_chunks * size_t(L.qrows) * 8);
+    L.sc_lse = take(slabs * size_t(L.qrows) * 4);
+    L.sc_tokimp = take(slabs * size_t(s.max_cap > 0 ? s.max_cap : 1) * 4);
+    L.sc_vbar = take(slabs * ms * kHeadDim * 4);
+    L.sc_z = take(slabs * ms * 4);
+    L.total = o;
+    return L;
+}
+
+int check_shape(const skipkv_shape* s);          // SKIPKV_OK or an error code
+int cuda_fail(cudaError_t e);                    // records the message, returns SKIPKV_ERR_CUDA
+int num_sms();
+
+#define SKIPKV_CUDA(expr)                                            \
+    do {                                                             \
+        cudaError_t e__ = (expr);                                    \
+        if (e__ != cudaSuccess) return ::skipkv::cuda_fail(e__);     \
+    } while (0)
+
+// ---------------------------------------------------------------------------------------
+// Device helpers
+// ---------------------------------------------------------------------------------------
+#ifdef __CUDACC__
+
+__device__ __forceinline__ size_t slab_row0(const int64_t* slab_off, const int32_t* cap, int Hk, int b, int h) {
+    return size_t(slab_off[b]) * Hk + size_t(h) * cap[b];
+}
+
+__device__ __forceinline__ float bf16lo(uint32_t x) { return __uint_as_float(x << 16); }
+__device__ __forceinline__ float bf16hi(uint32_t x) { return __uint_as_float(x & 0xffff0000u); }
+__device__ __forceinline__ float2 bf16x2_to_f2(uint32_t x) { return make_float2(bf16lo(x), bf16hi(x)); }
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+
+// ---- mbarrier + bulk asynchronous copies (TMA engine, untiled form) -------------------
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_fence_init() {
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait: returns false if the phase did not complete within the limit.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, uint32_t limit = (1u << 22)) {
+    for (uint32_t i = 0; i < limit; ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (i > 64) __nanosleep(64);
+    }
+    return false;
+}
+// global -> shared, completion counted in bytes on an mbarrier.  16-byte aligned, size % 16 == 0.
+__device__ __forceinline__ void bulk_g2s(void* smem_dst, const void* gsrc, uint32_t bytes, uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+            smem_u32(smem_dst)),
+        "l"(gsrc), "r"(bytes), "r"(smem_u32(bar))
+        : "memory");
+}
+// shared -> global, tracked by the issuing thread's bulk async-group.
+__device__ __forceinline__ void bulk_s2g(void* gdst, const void* smem_src, uint32_t bytes) {
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gdst),
+                 "r"(smem_u32(smem_src)), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read_all() {
+    asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
+
+#endif  // __CUDACC__
+
+}  // namespace skipkv

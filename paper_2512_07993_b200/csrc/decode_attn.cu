@@ -1,0 +1,428 @@
+// skipkv_decode_attn: GQA decode attention over the ragged, compacted cache (the attention
+// equation of paper Section 4.1 with one query per head), with the steering add of Section 4.2
+// performed by the tail of the same launch.
+//
+// The step is HBM bound: every live K and V row is read exactly once.  Design:
+//  * Work = 64-row tiles enumerated over all (sequence, head) slabs.  The tile list is cut into
+//    equal contiguous ranges, one per persistent CTA, so CTAs are balanced whatever the ragged
+//    lengths are; a CTA's range may cross slab boundaries, each (CTA, slab) intersection gives
+//    one partial result (running max, sum, 128-wide accumulator per head).
+//  * K and V tiles are streamed into a shared-memory ring with bulk asynchronous copies (each
+//    tile is one contiguous block of the slab) signalled through mbarriers, issued two tiles
+//    ahead by one elected lane; eight warps work on 8 rows of a tile each.  (256 threads per
+//    CTA and two CTAs per SM leave 128 registers per thread, which the mapping below needs.)
+//  * Consumer mapping: a half-warp per row, 8 channels (16 bytes) per lane.  The four heads of
+//    the group share every K/V load.  fp32 arithmetic with packed two-wide FMAs; the 16 partial
+//    dot products a lane holds for 4 rows x 4 heads are reduced with a 15-shuffle butterfly
+//    that leaves one finished logit per lane.
+//  * Softmax is online in base 2 (the log2(e)/sqrt(d) factor is folded into q).
+//  * The last CTA to deliver a partial for a slab (self-resetting counter in the workspace)
+//    merges that slab's partials and writes the bf16 output.
+//  * Every wait is bounded; on expiry the status word is flagged and the kernel drains.
+#include "common.cuh"
+#include "steer.cuh"
+
+namespace skipkv {
+
+constexpr int kTileRows = 64;
+constexpr int kTileBytes = kTileRows * kRowBytes;         // 16 KB for K, same for V
+constexpr int kStages = 3;
+constexpr int kConsWarps = 8;
+constexpr int kDecThreads = kConsWarps * 32;
+constexpr int kCtasPerSm = 2;
+constexpr int kPartStride = 130;                          // global record: 128 accumulators + max + sum
+constexpr int kWpStride = 132;                            // same record in shared memory, 16-byte aligned rows
+constexpr int kMaxDecSlabs = 8192;
+
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+struct DecSmem {
+    uint64_t full[kStages];
+    uint64_t empty[kStages];
+    int abort_flag;
+    int is_last;
+    uint32_t wsum[kDecThreads / 32];
+};
+
+__device__ __forceinline__ void consumer_bar() { asm volatile("bar.sync 1, %0;" ::"n"(kConsWarps * 32) : "memory"); }
+
+// One consumer warp, 8 rows [row_base, row_base+8) of a tile, heads hg*4 .. hg*4+3.
+template <bool kGuard>
+__device__ __forceinline__ void tile_rows(const uint8_t* Ks, const uint8_t* Vs, int row_base, int rows, int lane,
+                                          const float2 (&q2)[4][4], float2 (&acc)[4][4], float& m_run,
+                                          float& l_run) {
+    const int half = lane >> 4, l16 = lane & 15;
+    const uint4* Kp = reinterpret_cast<const uint4*>(Ks + size_t(row_base + half) * kRowBytes) + l16;
+    const uint4* Vp = reinterpret_cast<const uint4*>(Vs + size_t(row_base + half) * kRowBytes) + l16;
+    float part[16];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const uint4 kk = Kp[i * 32];                     // row_base + 2i + half
+        const float2 k0 = bf16x2_to_f2(kk.x), k1 = bf16x2_to_f2(kk.y), k2 = bf16x2_to_f2(kk.z),
+                     k3 = bf16x2_to_f2(kk.w);
+#pragma unroll
+        for (int h = 0; h < 4; ++h) {
+            float2 a = __fmul2_rn(q2[h][0], k0);
+            a = __ffma2_rn(q2[h][1], k1, a);
+            a = __ffma2_rn(q2[h][2], k2, a);
+            a = __ffma2_rn(q2[h][3], k3, a);
+            part[i * 4 + h] = a.x + a.y;
+        }
+    }
+    // butterfly over the 16 lanes of a half-warp: lane l16 ends with the full sum of part[l16]
+    const bool u8 = lane & 8, u4 = lane & 4, u2 = lane & 2, u1 = lane & 1;
+    float r8[8], r4[4], r2[2];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        const float mine = u8 ? part[k + 8] : part[k], send = u8 ? part[k] : part[k + 8];
+        r8[k] = mine + __shfl_xor_sync(0xffffffffu, send, 8);
+    }
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const float mine = u4 ? r8[k + 4] : r8[k], send = u4 ? r8[k] : r8[k + 4];
+        r4[k] = mine + __shfl_xor_sync(0xffffffffu, send, 4);
+    }
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+        const float mine = u2 ? r4[k + 2] : r4[k], send = u2 ? r4[k] : r4[k + 2];
+        r2[k] = mine + __shfl_xor_sync(0xffffffffu, send, 2);
+    }
+    float s;
+    {
+        const float mine = u1 ? r2[1] : r2[0], send = u1 ? r2[0] : r2[1];
+        s = mine + __shfl_xor_sync(0xffffffffu, send, 1);
+    }
+    // this lane's logit: row row_base + 2*(l16>>2) + half, head l16 & 3
+    if (kGuard) {
+        if (row_base + 2 * (l16 >> 2) + half >= rows) s = -INFINITY;
+    }
+    float bm = s;
+    bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 4));
+    bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 8));
+    bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 16));
+    const float m_new = fmaxf(m_run, bm);
+    if (__any_sync(0xffffffffu, m_new > m_run)) {
+        const float sc = ex2(m_run - m_new);             // first block: 2^(-inf) = 0
+        l_run *= sc;
+#pragma unroll
+        for (int h = 0; h < 4; ++h) {
+            const float sh = __shfl_sync(0xffffffffu, sc, h);
+            const float2 s2 = make_float2(sh, sh);
+#pragma unroll
+            for (int c = 0; c < 4; ++c) acc[h][c] = __fmul2_rn(acc[h][c], s2);
+        }
+        m_run = m_new;
+    }
+    const float p = ex2(s - m_run);
+    l_run += p;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        uint4 vv = Vp[i * 32];
+        if (kGuard) {
+            if (row_base + 2 * i + half >= rows) vv = make_uint4(0u, 0u, 0u, 0u);   // stale shared memory
+        }
+        const float2 v0 = bf16x2_to_f2(vv.x), v1 = bf16x2_to_f2(vv.y), v2 = bf16x2_to_f2(vv.z),
+                     v3 = bf16x2_to_f2(vv.w);
+#pragma unroll
+        for (int h = 0; h < 4; ++h) {
+            const float ph = __shfl_sync(0xffffffffu, p, (lane & 16) | (i * 4 + h));
+            const float2 pp = make_float2(ph, ph);
+            acc[h][0] = __ffma2_rn(pp, v0, acc[h][0]);
+            acc[h][1] = __ffma2_rn(pp, v1, acc[h][1]);
+            acc[h][2] = __ffma2_rn(pp, v2, acc[h][2]);
+            acc[h][3] = __ffma2_rn(pp, v3, acc[h][3]);
+        }
+    }
+}
+
+__global__ void __launch_bounds__(kDecThreads, kCtasPerSm)
+decode_attn_kernel(int batch, int Hq, int Hk, int n_slabs, const int64_t* slab_off, const int32_t* cap,
+                   const __nv_bfloat16* q, const uint8_t* K, const uint8_t* V, const int32_t* kv_len,
+                   __nv_bfloat16* out, uint32_t* status, uint32_t* dec_cnt, float* dec_part, int d_model,
+                   __nv_bfloat16* hidden, const __nv_bfloat16* steer_vec, const float* alpha, const uint8_t* flag) {
+    extern __shared__ __align__(1024) uint8_t dsm[];
+    uint8_t* ring = dsm;                                                     // kStages x (K tile, V tile)
+    float* wpart = reinterpret_cast<float*>(dsm + kStages * 2 * kTileBytes);  // [8 warps][4 heads][132]
+    DecSmem* sm = reinterpret_cast<DecSmem*>(wpart + kConsWarps * 4 * kWpStride);
+    int* pref = reinterpret_cast<int*>(sm + 1);                              // [n_slabs + 1] tile prefix
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    auto live = [&](int s) { return min(max(kv_len[s], 0), cap[s / Hk]); };   // live rows of slab s
+    const int n = Hq / Hk;                     // heads per group
+    const int NG = (n + 3) / 4;                // head groups of 4 (1 or 2)
+    const int G = gridDim.x, cta = blockIdx.x;
+
+    if (tid == 0) {
+        for (int s = 0; s < kStages; ++s) { mbar_init(&sm->full[s], 1); mbar_init(&sm->empty[s], kConsWarps); }
+        sm->abort_flag = 0;
+        sm->is_last = 0;
+        mbar_fence_init();
+    }
+    // tile prefix over slabs (block scan; every thread owns a contiguous block of slabs)
+    {
+        const int per = (n_slabs + kDecThreads - 1) / kDecThreads;
+        const int s0 = min(tid * per, n_slabs), s1 = min(s0 + per, n_slabs);
+        uint32_t local = 0;
+        for (int s = s0; s < s1; ++s) local += uint32_t((live(s) + kTileRows - 1) / kTileRows);
+        // inclusive warp scan, then across warps
+        uint32_t inc = local;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const uint32_t a = __shfl_up_sync(0xffffffffu, inc, d);
+            if (lane >= d) inc += a;
+        }
+        if (lane == 31) sm->wsum[warp] = inc;
+        __syncthreads();                               // also publishes the barrier inits
+        uint32_t base = 0;
+        for (int w = 0; w < warp; ++w) base += sm->wsum[w];
+        uint32_t run = base + inc - local;
+        for (int s = s0; s < s1; ++s) {
+            pref[s] = int(run);
+            run += uint32_t((live(s) + kTileRows - 1) / kTileRows);
+        }
+        if (tid == kDecThreads - 1) pref[n_slabs] = int(run);
+        __syncthreads();
+    }
+    const int Ttot = pref[n_slabs];
+    const int per_cta = max(1, (Ttot + G - 1) / G);
+    const int t_begin = min(cta * per_cta, Ttot), t_end = min(t_begin + per_cta, Ttot);
+
+    // slab holding tile t_begin: largest s with pref[s] <= t_begin and a non-empty slab
+    int slab0 = 0;
+    if (t_begin < t_end) {
+        int lo = 0, hi = n_slabs - 1;
+        while (lo < hi) {
+            const int mid = (lo + hi + 1) >> 1;
+            if (pref[mid] <= t_begin) lo = mid; else hi = mid - 1;
+        }
+        slab0 = lo;
+    }
+
+    {
+        // ------------------------------------------------------------------ consumers
+        const int hg = warp % NG;                       // head group of this warp
+        const int rb = warp / NG;                       // row block: rows [rb*NG*8, (rb+1)*NG*8) of each tile
+        const int half = lane >> 4, l16 = lane & 15;
+        const float qscale = 1.4426950408889634f * rsqrtf(float(kHeadDim));
+        float2 q2[4][4], acc[4][4];
+        float m_run = -INFINITY, l_run = 0.f;
+        int slab = slab0, consumed = 0;
+        bool seg_open = false;
+        bool aborted = false;
+        // copy issue (warp 0, lane 0 only): tile k of this CTA goes to stage k % kStages
+        const bool is_producer = (tid == 0);
+        int p_slab = slab0, issued = 0;
+        auto issue_next = [&]() {
+            const int tt = t_begin + issued;
+            if (tt >= t_end) return;
+            while (pref[p_slab + 1] <= tt) ++p_slab;
+            const int stage = issued % kStages, use = issued / kStages;
+            if (use > 0) {
+                if (sm->abort_flag || !mbar_wait(&sm->empty[stage], uint32_t(use - 1) & 1u)) {
+                    if (!sm->abort_flag) atomicOr(status, SKIPKV_STATUS_COPY_TIMEOUT);
+                    sm->abort_flag = 1;
+                    return;
+                }
+            }
+            const int pb = p_slab / Hk, ph = p_slab % Hk;
+            const int j = tt - pref[p_slab];
+            const int rows = min(kTileRows, live(p_slab) - j * kTileRows);
+            const size_t off = (slab_row0(slab_off, cap, Hk, pb, ph) + size_t(j) * kTileRows) * kRowBytes;
+            const uint32_t bytes = uint32_t(rows) * kRowBytes;
+            uint8_t* dstK = ring + size_t(stage) * 2 * kTileBytes;
+            mbar_expect_tx(&sm->full[stage], 2 * bytes);
+            bulk_g2s(dstK, K + off, bytes, &sm->full[stage]);
+            bulk_g2s(dstK + kTileBytes, V + off, bytes, &sm->full[stage]);
+            ++issued;
+        };
+        if (is_producer)
+            for (int k = 0; k < kStages - 1; ++k) issue_next();
+        for (int t = t_begin; t < t_end; ++t, ++consumed) {
+            if (is_producer && !sm->abort_flag) issue_next();       // keeps kStages-1 tiles in flight
+            while (pref[slab + 1] <= t) ++slab;
+            const int b = slab / Hk, h = slab % Hk;
+            if (!seg_open) {
+                // new (CTA, slab) segment: load the group's queries, reset the running state
+#pragma unroll
+                for (int hh = 0; hh < 4; ++hh) {
+                    const int hl = hg * 4 + hh;
+                    uint4 qq = make_uint4(0u, 0u, 0u, 0u);
+                    if (hl < n)
+                        qq = reinterpret_cast<const uint4*>(q + (size_t(b) * Hq + size_t(h) * n + hl) * kHeadDim)[l16];
+                    const float2 s2 = make_float2(qscale, qscale);
+                    q2[hh][0] = __fmul2_rn(bf16x2_to_f2(qq.x), s2);
+                    q2[hh][1] = __fmul2_rn(bf16x2_to_f2(qq.y), s2);
+                    q2[hh][2] = __fmul2_rn(bf16x2_to_f2(qq.z), s2);
+                    q2[hh][3] = __fmul2_rn(bf16x2_to_f2(qq.w), s2);
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) acc[hh][c] = make_float2(0.f, 0.f);
+                }
+                m_run = -INFINITY;
+                l_run = 0.f;
+                seg_open = true;
+            }
+            const int stage = consumed % kStages, use = consumed / kStages;
+            const int j = t - pref[slab];
+            const int rows = min(kTileRows, live(slab) - j * kTileRows);
+            if (!aborted) {
+                if (sm->abort_flag || !mbar_wait(&sm->full[stage], uint32_t(use) & 1u)) {
+                    if (!sm->abort_flag) atomicOr(status, SKIPKV_STATUS_COPY_TIMEOUT);
+                    sm->abort_flag = 1;
+                    aborted = true;
+                }
+            }
+            if (!aborted) {
+                const uint8_t* Ks = ring + size_t(stage) * 2 * kTileBytes;
+                const uint8_t* Vs = Ks + kTileBytes;
+                for (int sub = 0; sub < NG; ++sub) {
+                    const int row_base = (rb * NG + sub) * 8;
+                    if (row_base >= rows) break;
+                    if (rows == kTileRows) tile_rows<false>(Ks, Vs, row_base, rows, lane, q2, acc, m_run, l_run);
+                    else tile_rows<true>(Ks, Vs, row_base, rows, lane, q2, acc, m_run, l_run);
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sm->empty[stage]);
+            }
+            const bool seg_end = (t + 1 == t_end) || (pref[slab + 1] <= t + 1);
+            if (!seg_end) continue;
+
+            // ---------------------------------------------------------- flush this (CTA, slab) segment
+            seg_open = false;
+            // halves of the warp hold different rows: add them; finish the sum of p
+#pragma unroll
+            for (int hh = 0; hh < 4; ++hh)
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    acc[hh][c].x += __shfl_xor_sync(0xffffffffu, acc[hh][c].x, 16);
+                    acc[hh][c].y += __shfl_xor_sync(0xffffffffu, acc[hh][c].y, 16);
+                }
+            l_run += __shfl_xor_sync(0xffffffffu, l_run, 4);
+            l_run += __shfl_xor_sync(0xffffffffu, l_run, 8);
+            l_run += __shfl_xor_sync(0xffffffffu, l_run, 16);
+            float* wp = wpart + size_t(warp) * 4 * kWpStride;
+            if (half == 0) {
+#pragma unroll
+                for (int hh = 0; hh < 4; ++hh) {
+                    float4* dst = reinterpret_cast<float4*>(wp + hh * kWpStride + l16 * 8);
+                    dst[0] = make_float4(acc[hh][0].x, acc[hh][0].y, acc[hh][1].x, acc[hh][1].y);
+                    dst[1] = make_float4(acc[hh][2].x, acc[hh][2].y, acc[hh][3].x, acc[hh][3].y);
+                }
+            }
+            if (lane < 4) {
+                wp[lane * kWpStride + 128] = m_run;
+                wp[lane * kWpStride + 129] = l_run;
+            }
+            consumer_bar();
+            // merge the warps of each head group; thread -> (head, channel) pairs
+            const int fc = pref[slab] / per_cta, lc = (pref[slab + 1] - 1) / per_cta;
+            const int n_part = lc - fc + 1;
+            __nv_bfloat16* o = out + (size_t(b) * Hq + size_t(h) * n) * kHeadDim;
+            float* rec = dec_part + size_t(cta + slab) * n * kPartStride;
+            for (int idx = tid; idx < n * kHeadDim; idx += kConsWarps * 32) {
+                const int hl = idx / kHeadDim, c = idx % kHeadDim;
+                const int g2 = hl / 4, hh = hl % 4;
+                float M = -INFINITY;
+                for (int w = g2; w < kConsWarps; w += NG) M = fmaxf(M, wpart[(w * 4 + hh) * kWpStride + 128]);
+                float L = 0.f, A = 0.f;
+                for (int w = g2; w < kConsWarps; w += NG) {
+                    const float* p = wpart + (w * 4 + hh) * kWpStride;
+                    const float e = ex2(p[128] - M);
+                    L += p[129] * e;
+                    A += p[c] * e;
+                }
+                if (n_part == 1) {
+                    o[idx] = __float2bfloat16_rn(L > 0.f ? A / L : 0.f);
+                } else {
+                    rec[hl * kPartStride + c] = A;
+                    if (c == 0) { rec[hl * kPartStride + 128] = M; rec[hl * kPartStride + 129] = L; }
+                }
+            }
+            if (n_part > 1) {
+                __threadfence();
+                consumer_bar();
+                if (tid == 0) {
+                    const uint32_t old = atomicAdd(dec_cnt + slab, 1u);
+                    const int last = (old == uint32_t(n_part - 1)) ? 1 : 0;
+                    if (last) dec_cnt[slab] = 0u;          // self-resetting for the next launch
+                    sm->is_last = last;
+                }
+                consumer_bar();
+                if (sm->is_last) {
+                    __threadfence();
+                    const float* r0 = dec_part + size_t(fc + slab) * n * kPartStride;
+                    for (int idx = tid; idx < n * kHeadDim; idx += kConsWarps * 32) {
+                        const int hl = idx / kHeadDim, c = idx % kHeadDim;
+                        float M = -INFINITY;
+                        for (int p = 0; p < n_part; ++p)
+                            M = fmaxf(M, __ldcg(r0 + (size_t(p) * n + hl) * kPartStride + 128));
+                        float L = 0.f, A = 0.f;
+                        for (int p = 0; p < n_part; ++p) {
+                            const float* rp = r0 + (size_t(p) * n + hl) * kPartStride;
+                            const float e = ex2(__ldcg(rp + 128) - M);
+                            L += __ldcg(rp + 129) * e;
+                            A += __ldcg(rp + c) * e;
+                        }
+                        o[idx] = __float2bfloat16_rn(L > 0.f ? A / L : 0.f);
+                    }
+                }
+            }
+            consumer_bar();                                // wpart and is_last reusable
+        }
+        // drain (only after an abort can copies still be in flight): they must land before exit
+        if (is_producer)
+            for (int k = consumed; k < issued; ++k) mbar_wait(&sm->full[k % kStages], uint32_t(k / kStages) & 1u);
+        // slabs with no live row: zeros (owned round-robin)
+        for (int s = cta; s < n_slabs; s += G) {
+            if (live(s) > 0) continue;
+            const int b = s / Hk, h = s % Hk;
+            __nv_bfloat16* o = out + (size_t(b) * Hq + size_t(h) * n) * kHeadDim;
+            for (int idx = tid; idx < n * kHeadDim; idx += kConsWarps * 32) o[idx] = __float2bfloat16_rn(0.f);
+        }
+    }
+    // ---------------------------------------------------------------------- steering epilogue
+    if (hidden != nullptr) {
+        const int vec_per_row = d_model / 8, total = batch * vec_per_row;
+        for (int i = cta * kDecThreads + tid; i < total; i += G * kDecThreads)
+            steer_vec8(i, vec_per_row, hidden, steer_vec, alpha, flag);
+    }
+}
+
+}  // namespace skipkv
+
+using namespace skipkv;
+
+extern "C" int skipkv_decode_attn(const skipkv_shape* shape, const void* q, const void* K, const void* V,
+                                  const int32_t* kv_len, void* out, void* hidden, const void* steer_vec,
+                                  const float* alpha, const uint8_t* flag, void* ws, void* stream) {
+    if (int rc = check_shape(shape)) return rc;
+    if (!q || !K || !V || !kv_len || !out) return SKIPKV_ERR_INVALID_ARG;
+    if (hidden && (!steer_vec || !alpha || !flag || shape->d_model <= 0)) return SKIPKV_ERR_INVALID_ARG;
+    if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255)) return SKIPKV_ERR_WORKSPACE;
+    if ((reinterpret_cast<uintptr_t>(K) & 15) || (reinterpret_cast<uintptr_t>(V) & 15) ||
+        (reinterpret_cast<uintptr_t>(q) & 15))
+        return SKIPKV_ERR_INVALID_ARG;
+    const WsLayout L = make_layout(*shape);
+    if (L.slabs > kMaxDecSlabs) return SKIPKV_ERR_UNSUPPORTED;
+    uint8_t* w = static_cast<uint8_t*>(ws);
+    const size_t smem = size_t(kStages) * 2 * kTileBytes + size_t(kConsWarps) * 4 * kWpStride * 4 + sizeof(DecSmem) +
+                        size_t(L.slabs + 1) * 4;
+    static thread_local size_t attr_smem = 0;
+    if (smem > attr_smem) {
+        SKIPKV_CUDA(cudaFuncSetAttribute(decode_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
+        attr_smem = smem;
+    }
+    int grid = num_sms() * kCtasPerSm;
+    if (grid > L.dec_max_ctas) grid = L.dec_max_ctas;
+    decode_attn_kernel<<<grid, kDecThreads, smem, static_cast<cudaStream_t>(stream)>>>(
+        shape->batch, shape->n_q_heads, shape->n_kv_heads, L.slabs, shape->slab_off, shape->cap,
+        static_cast<const __nv_bfloat16*>(q), static_cast<const uint8_t*>(K), static_cast<const uint8_t*>(V), kv_len,
+        static_cast<__nv_bfloat16*>(out), &reinterpret_cast<Header*>(w + L.header)->status,
+        reinterpret_cast<uint32_t*>(w + L.dec_cnt), reinterpret_cast<float*>(w + L.dec_part), shape->d_model,
+        static_cast<__nv_bfloat16*>(hidden), static_cast<const __nv_bfloat16*>(steer_vec), alpha, flag);
+    SKIPKV_CUDA(cudaGetLastError());
+    return SKIPKV_OK;
+}

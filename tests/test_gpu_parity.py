@@ -1,0 +1,344 @@
+"""GPU parity: every step of the CUDA path, called through the C ABI, against the CPU oracle
+on the same seeded inputs.
+
+Tolerance contract
+  * keep flags, kept indices, index maps, range tables, moved K/V rows, steering: bit-exact
+  * fp32 importance / redundancy / lambda / score: rtol 1e-3 (components compared separately)
+  * decode attention: max error <= 2e-2 of the row's largest |output| (bf16 output)
+Selection from float scores is checked in three parts: the GPU's selection equals the
+oracle's selection rule applied to the GPU's own scores; fed the oracle's scores it equals
+the oracle's selection; and end to end the keep sets agree except in slabs where the oracle's
+scores around the cut are closer than 1e-5 relative (counted, and required to be zero here).
+"""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2512_07993_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2512_07993_b200 import build, binding
+    build.build()
+    binding.lib()
+    return binding
+
+
+def oshape(L):
+    cfg = L["cfg"]
+    return dict(batch=cfg.batch, Hq=cfg.n_q_heads, Hk=cfg.n_kv_heads, d=cfg.head_dim, alpha=cfg.window,
+                max_sent=L["max_sent"], slab_off=L["slab_off"], cap=L["cap"])
+
+
+def oracle_scores(L, want_tok=True):
+    return oracle.score_batch(oshape(L), W.bf16_bits(L["K"]), W.bf16_bits(L["q_win"]), L["kv_len"], L["sent_off"],
+                              L["n_sent"], float(np.float32(0.1)), float(np.float32(0.95)), float(np.float32(1e-6)),
+                              want_tok_imp=want_tok)
+
+
+def cases():
+    return {
+        "smoke": W.config(0),
+        "tiny": W.config(1),
+        "ragged": W.config(1, name="ragged", batch=3, ctx_lo=700, ctx_hi=2100, budget=1500, seed=77, dup_rate=0.3),
+        "group5": W.config(0, name="group5", n_q_heads=10, n_kv_heads=2, window=12, ctx_lo=500, ctx_hi=900,
+                           budget=333, seed=5),
+    }
+
+
+@pytest.fixture(scope="module", params=list(cases().keys()))
+def case(request, B):
+    L = W.make_layer(cases()[request.param])
+    return L, oracle_scores(L)
+
+
+def assert_close(name, got, ref, rtol=1e-3, atol=0.0):
+    got = np.asarray(got, np.float64); ref = np.asarray(ref, np.float64)
+    err = np.abs(got - ref) - (atol + rtol * np.abs(ref))
+    assert (err <= 0).all(), f"{name}: worst excess {err.max():.3e} at {np.unravel_index(err.argmax(), err.shape)}"
+
+
+def live_mask(L):
+    ms = L["max_sent"]
+    return np.arange(ms)[None, None, :] < L["n_sent"][:, :, None]
+
+
+# ----------------------------------------------------------------------------- score
+def test_score_matches_oracle(B, case):
+    L, ref = case
+    D = B.DeviceLayer(L)
+    D.score()
+    torch.cuda.synchronize()
+    assert D.status() == 0
+    m = live_mask(L)
+    imp, red, lam, sc = (x.cpu().numpy() for x in (D.sent_imp, D.sent_red, D.sent_lam, D.sent_score))
+    assert_close("sent_imp", imp[m], ref["imp"][m])
+    assert_close("sent_red", red[m], ref["red"][m])
+    assert ((lam[m] == 0) == (ref["lam"][m] == 0)).all(), "redundant set differs"
+    assert_close("sent_lam", lam[m], ref["lam"][m])
+    assert_close("sent_score", sc[m], ref["score"][m], rtol=1e-3, atol=1e-6)
+    tok = D.tok_imp.cpu().numpy()
+    cfg = L["cfg"]
+    for b in range(cfg.batch):
+        for h in range(cfg.n_kv_heads):
+            sl = W.slab_rows(L, b, h)
+            n = int(L["kv_len"][b, h])
+            assert_close(f"tok_imp[{b},{h}]", tok[sl][:n], ref["tok_imp"][sl][:n])
+
+
+# ----------------------------------------------------------------------------- select
+def near_tie_slabs(L, score, sel, rel=1e-5):
+    """Slabs whose oracle scores at ranks k*..k*+2 (the cut neighbourhood) are closer than rel."""
+    cfg = L["cfg"]
+    out = set()
+    for b in range(cfg.batch):
+        for h in range(cfg.n_kv_heads):
+            S = int(L["n_sent"][b, h])
+            if int(L["kv_len"][b, h]) <= cfg.budget:
+                continue
+            off = L["sent_off"][b, h]
+            total = off[S]
+            forced = off[1:S + 1] > total - cfg.window
+            s = score[b, h, :S][~forced]
+            order = np.argsort(-s, kind="stable")
+            kstar = int(sel["keep"][b, h, :S][~forced].sum())
+            nb = s[order[max(kstar - 1, 0):kstar + 3]]
+            for i in range(len(nb)):
+                for j in range(i + 1, len(nb)):
+                    if abs(nb[i] - nb[j]) <= rel * max(abs(nb[i]), abs(nb[j])):
+                        out.add((b, h))
+    return out
+
+
+def test_select_three_part_contract(B, case):
+    L, ref = case
+    cfg = L["cfg"]
+    D = B.DeviceLayer(L)
+    # (ii) the selection rule itself is exact: oracle scores in, oracle keep out
+    D.sent_score.copy_(torch.from_numpy(ref["score"]))
+    D.select()
+    torch.cuda.synchronize()
+    sel = oracle.select_batch(ref["score"], L["sent_off"], L["n_sent"], cfg.budget, cfg.window)
+    assert np.array_equal(D.keep.cpu().numpy(), sel["keep"])
+    assert np.array_equal(D.n_kept.cpu().numpy(), sel["n_kept"])
+    assert np.array_equal(D.new_len.cpu().numpy(), sel["new_len"])
+    assert np.array_equal(D.kept_idx.cpu().numpy(), sel["kept_idx"])
+    over = L["kv_len"] > cfg.budget
+    assert (sel["new_len"][over] <= cfg.budget).all()
+    # (i) GPU selection == oracle rule on the GPU's own scores
+    D.score(); D.select()
+    torch.cuda.synchronize()
+    gs = D.sent_score.cpu().numpy()
+    gs[~live_mask(L)] = 0
+    sel_g = oracle.select_batch(gs, L["sent_off"], L["n_sent"], cfg.budget, cfg.window)
+    assert np.array_equal(D.keep.cpu().numpy(), sel_g["keep"])
+    assert np.array_equal(D.new_len.cpu().numpy(), sel_g["new_len"])
+    # (iii) end to end, excusing only near ties at the cut
+    excused = near_tie_slabs(L, ref["score"], sel)
+    keep_g = D.keep.cpu().numpy()
+    for b in range(cfg.batch):
+        for h in range(cfg.n_kv_heads):
+            if (b, h) in excused:
+                continue
+            assert np.array_equal(keep_g[b, h], sel["keep"][b, h]), (b, h)
+    if cfg.name == "tiny":                      # the reference configuration must need no excuse
+        assert len(excused) == 0, f"near-tie slabs: {sorted(excused)}"
+    assert len(excused) <= 0.1 * cfg.batch * cfg.n_kv_heads, f"near-tie slabs: {sorted(excused)}"
+    assert D.status() == 0
+
+
+def test_select_edge_cases(B):
+    cfg = W.config(0, ctx_lo=200, ctx_hi=260)
+    L = W.make_layer(cfg)
+    D = B.DeviceLayer(L)
+    ms = L["max_sent"]
+    rng = np.random.default_rng(1)
+    score = np.round(rng.standard_normal((cfg.batch, cfg.n_kv_heads, ms)), 1).astype(np.float32)   # many exact ties
+    score[0, 0, :4] = [0.0, -0.0, 0.0, -0.0]
+    for budget, pt in [(0, 0), (1, 0), (50, 0), (50, 8), (120, 300), (10_000, 8), (97, 1)]:
+        D.params = B.make_params(0.1, 0.95, 1e-6, budget, pt)
+        D.sent_score.copy_(torch.from_numpy(score))
+        D.select()
+        torch.cuda.synchronize()
+        sel = oracle.select_batch(score, L["sent_off"], L["n_sent"], budget, pt)
+        assert np.array_equal(D.keep.cpu().numpy(), sel["keep"]), (budget, pt)
+        assert np.array_equal(D.kept_idx.cpu().numpy(), sel["kept_idx"]), (budget, pt)
+        assert np.array_equal(D.new_len.cpu().numpy(), sel["new_len"]), (budget, pt)
+
+
+# ----------------------------------------------------------------------------- compact
+def run_compact_case(B, L, keep):
+    cfg = L["cfg"]
+    D = B.DeviceLayer(L)
+    D.keep.copy_(torch.from_numpy(keep))
+    D.K[:] = L["K"].cuda(); D.V[:] = L["V"].cuda()
+    D.compact()
+    torch.cuda.synchronize()
+    assert D.status() == 0
+    ref = oracle.compact_batch(oshape(L), W.bf16_bits(L["K"]), W.bf16_bits(L["V"]), keep, L["sent_off"],
+                               L["sent_id"], L["n_sent"], L["kv_len"])
+    assert np.array_equal(D.kv_len.cpu().numpy(), ref["kv_len"])
+    assert np.array_equal(D.n_sent.cpu().numpy(), ref["n_sent"])
+    assert np.array_equal(D.sent_off.cpu().numpy(), ref["sent_off"])
+    assert np.array_equal(D.sent_id.cpu().numpy(), ref["sent_id"])
+    Kg, Vg, im = W.bf16_bits(D.K.cpu()), W.bf16_bits(D.V.cpu()), D.index_map.cpu().numpy()
+    for b in range(cfg.batch):
+        for h in range(cfg.n_kv_heads):
+            sl = W.slab_rows(L, b, h)
+            n = int(ref["kv_len"][b, h])
+            assert np.array_equal(Kg[sl][:n], ref["K"][sl][:n]), (b, h)
+            assert np.array_equal(Vg[sl][:n], ref["V"][sl][:n]), (b, h)
+            assert np.array_equal(im[sl][:n], ref["index_map"][sl][:n]), (b, h)
+            assert (np.diff(im[sl][:n]) > 0).all()
+    return D, ref
+
+
+def test_compact_matches_oracle(B, case):
+    L, ref = case
+    cfg = L["cfg"]
+    sel = oracle.select_batch(ref["score"], L["sent_off"], L["n_sent"], cfg.budget, cfg.window)
+    run_compact_case(B, L, sel["keep"])
+
+
+def test_compact_patterns(B):
+    cfg = W.config(1, batch=2, ctx_lo=1500, ctx_hi=2048, seed=31)
+    L = W.make_layer(cfg)
+    ms = L["max_sent"]
+    rng = np.random.default_rng(2)
+    live = live_mask(L)
+    patterns = {
+        "all": np.ones((cfg.batch, cfg.n_kv_heads, ms), np.uint8),
+        "none": np.zeros((cfg.batch, cfg.n_kv_heads, ms), np.uint8),
+        "random": (rng.random((cfg.batch, cfg.n_kv_heads, ms)) < 0.5).astype(np.uint8),
+        "dense": (rng.random((cfg.batch, cfg.n_kv_heads, ms)) < 0.95).astype(np.uint8),   # many multi-segment moves by a few rows
+        "tail": (np.arange(ms)[None, None, :] >= ms // 2).astype(np.uint8) * np.ones((cfg.batch, cfg.n_kv_heads, 1), np.uint8),
+        "alternate": (np.arange(ms) % 2).astype(np.uint8)[None, None, :] * np.ones((cfg.batch, cfg.n_kv_heads, 1), np.uint8),
+    }
+    for name, keep in patterns.items():
+        keep = keep * live
+        run_compact_case(B, L, keep.astype(np.uint8))
+
+
+# ----------------------------------------------------------------------------- decode attention + steer
+def decode_err(out_bits, ref64):
+    got = W.bits_to_bf16(out_bits).float().numpy().astype(np.float64)
+    scale = np.abs(ref64).max(axis=-1, keepdims=True)
+    scale[scale == 0] = 1.0
+    return (np.abs(got - ref64) / scale).max()
+
+
+def test_decode_attn_full_and_ragged(B, case):
+    L, _ = case
+    cfg = L["cfg"]
+    rng = np.random.default_rng(3)
+    for mode in ("full", "ragged"):
+        kv_len = L["kv_len"].copy()
+        if mode == "ragged":
+            kv_len = rng.integers(0, L["kv_len"] + 1).astype(np.int32)
+            kv_len[0, 0] = 0                                   # an empty slab gives zeros
+            kv_len[-1, -1] = 1
+        D = B.DeviceLayer(L)
+        D.kv_len.copy_(torch.from_numpy(kv_len))
+        hid0 = D.hidden.clone()
+        D.decode_attn(steer=True)
+        torch.cuda.synchronize()
+        assert D.status() == 0
+        _, o64 = oracle.decode_attn_batch(oshape(L), W.bf16_bits(L["q"]), W.bf16_bits(L["K"]), W.bf16_bits(L["V"]),
+                                          kv_len)
+        err = decode_err(W.bf16_bits(D.out.cpu()), o64)
+        assert err <= 2e-2, (mode, err)
+        if mode == "ragged":
+            g = cfg.group
+            assert not D.out[0, :g].float().abs().max().item()
+        # fused steering add: bit-exact, flagged rows only
+        ref_h = oracle.steer(W.bf16_bits(L["hidden"]), W.bf16_bits(L["steer_vec"]), L["alpha"], L["flag"])
+        assert np.array_equal(W.bf16_bits(D.hidden.cpu()), ref_h)
+        assert not torch.equal(D.hidden, hid0)
+        # a second launch on the same workspace (self-resetting counters) gives the same output
+        first = D.out.clone()
+        D.decode_attn(steer=False)
+        torch.cuda.synchronize()
+        assert torch.equal(first, D.out)
+
+
+def test_steer_standalone(B):
+    L = W.make_layer(W.config(0, d_model=4096, batch=5))
+    D = B.DeviceLayer(L)
+    B.skipkv_steer(L["cfg"].batch, L["cfg"].d_model, D.hidden, D.steer_vec, D.alpha, D.flag)
+    torch.cuda.synchronize()
+    ref = oracle.steer(W.bf16_bits(L["hidden"]), W.bf16_bits(L["steer_vec"]), L["alpha"], L["flag"])
+    assert np.array_equal(W.bf16_bits(D.hidden.cpu()), ref)
+
+
+# ----------------------------------------------------------------------------- whole path, device resident
+def test_whole_path_end_to_end(B, case):
+    L, ref = case
+    cfg = L["cfg"]
+    D = B.DeviceLayer(L)
+    D.score(); D.select(); D.compact(); D.decode_attn(steer=True)
+    torch.cuda.synchronize()
+    assert D.status() == 0
+    sel = oracle.select_batch(ref["score"], L["sent_off"], L["n_sent"], cfg.budget, cfg.window)
+    cmp_ = oracle.compact_batch(oshape(L), W.bf16_bits(L["K"]), W.bf16_bits(L["V"]), sel["keep"], L["sent_off"],
+                                L["sent_id"], L["n_sent"], L["kv_len"])
+    assert np.array_equal(D.keep.cpu().numpy(), sel["keep"])
+    assert np.array_equal(D.kv_len.cpu().numpy(), cmp_["kv_len"])
+    assert (cmp_["kv_len"] <= np.maximum(cfg.budget, L["kv_len"] * (L["kv_len"] <= cfg.budget))).all()
+    Kg = W.bf16_bits(D.K.cpu())
+    for b in range(cfg.batch):
+        for h in range(cfg.n_kv_heads):
+            sl = W.slab_rows(L, b, h)
+            n = int(cmp_["kv_len"][b, h])
+            assert np.array_equal(Kg[sl][:n], cmp_["K"][sl][:n])
+    _, o64 = oracle.decode_attn_batch(oshape(L), W.bf16_bits(L["q"]), cmp_["K"], cmp_["V"], cmp_["kv_len"])
+    assert decode_err(W.bf16_bits(D.out.cpu()), o64) <= 2e-2
+    # idempotent: a second eviction pass on the compacted cache keeps everything
+    D.score(); D.select()
+    torch.cuda.synchronize()
+    assert np.array_equal(D.new_len.cpu().numpy(), cmp_["kv_len"])
+
+
+def test_append_then_decode(B):
+    cfg = W.config(0, cap_extra=8)
+    L = W.make_layer(cfg)
+    D = B.DeviceLayer(L)
+    g = torch.Generator().manual_seed(4)
+    Kh, Vh = L["K"].clone(), L["V"].clone()
+    kv_len = L["kv_len"].copy()
+    for step in range(3):
+        k_new = torch.randn(cfg.batch, cfg.n_kv_heads, 128, generator=g).to(torch.bfloat16)
+        v_new = torch.randn(cfg.batch, cfg.n_kv_heads, 128, generator=g).to(torch.bfloat16)
+        B.skipkv_append(D.shape, D.K, D.V, k_new.cuda(), v_new.cuda(), D.kv_len, D.ws)
+        for b in range(cfg.batch):
+            for h in range(cfg.n_kv_heads):
+                r = W.slab_rows(L, b, h).start + int(kv_len[b, h])
+                Kh[r] = k_new[b, h]; Vh[r] = v_new[b, h]
+        kv_len += 1
+    torch.cuda.synchronize()
+    assert np.array_equal(D.kv_len.cpu().numpy(), kv_len)
+    assert torch.equal(D.K.cpu(), Kh) and torch.equal(D.V.cpu(), Vh)
+    D.decode_attn(steer=False)
+    torch.cuda.synchronize()
+    _, o64 = oracle.decode_attn_batch(oshape(L), W.bf16_bits(L["q"]), W.bf16_bits(Kh), W.bf16_bits(Vh), kv_len)
+    assert decode_err(W.bf16_bits(D.out.cpu()), o64) <= 2e-2
+
+
+def test_argument_errors(B):
+    L = W.make_layer(W.config(0))
+    D = B.DeviceLayer(L)
+    bad = B.make_shape(2, 8, 2, 64, 8, 256, D.max_sent, 512, D.slab_off, D.cap)     # head_dim 64
+    with pytest.raises(B.SkipKVError) as e:
+        B.skipkv_workspace_bytes(bad)
+    assert e.value.code == -2
+    bad = B.make_shape(2, 7, 2, 128, 8, 256, D.max_sent, 512, D.slab_off, D.cap)    # Hq % Hk != 0
+    with pytest.raises(B.SkipKVError):
+        B.skipkv_workspace_bytes(bad)
+    with pytest.raises(B.SkipKVError) as e:                                       # misaligned workspace
+        B.skipkv_decode_attn(D.shape, D.q, D.K, D.V, D.kv_len, D.out, None, None, None, None, D.ws[8:])
+    assert e.value.code == -3
