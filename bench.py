@@ -1,0 +1,331 @@
+#!/usr/bin/env python
+"""Benchmark of the SkipKV hot path on B200: one step = score + select + compact + decode
+attention (with the fused steering add) over one layer of the Llama-8B-shaped workload
+(batch 10, 8 KV / 32 query heads, head_dim 128, ragged 16K-32K cached tokens, budget 4096).
+
+    python bench.py --gpus N --steps K --warmup W          # this library (CUDA path)
+    python bench.py --impl reference ...                   # the CPU oracle on the host cores
+
+Prints ONE JSON line.  `value` is the eviction time (score+select+compact) per layer in
+microseconds with inputs resident in HBM; the decode-attention bandwidth and the per-step
+rooflines ride along in the same line.  With N > 1 every rank runs an independent replica of
+the workload (the path has no exchange step); the time is the max over ranks and the value is
+that time divided by the N layers processed.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2512_07993_b200 import workloads as W  # noqa: E402
+
+METRIC = "SkipKV compress+compact µs/layer and decode-attn HBM GB/s, 32K ctx, batch 10"
+UNIT = "us/layer (score+select+compact); decode-attn GB/s in decode_attn_gbs"
+LAUNCHES_PER_STEP = {"score": 6, "select": 1, "compact": 2, "decode_attn": 1}
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return dict(hbm_gbs=float(d["hbm_gbs"]), bf16_tflops=float(d.get("bf16_tflops", 0.0)), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, source="fallback")
+
+
+def ncu_traffic():
+    """DRAM bytes per launch from the committed ncu summaries (None when not captured)."""
+    p = os.path.join(ROOT, "profiles", "dram_traffic.json")
+    return json.load(open(p)) if os.path.exists(p) else {}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.lines, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-i", str(self.index), "-lms", "100"], stdout=subprocess.PIPE, text=True)
+            threading.Thread(target=self._pump, daemon=True).start()
+        except Exception:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.time(), line.strip()))
+
+    def stop(self, t0, t1):
+        if self.proc is None:
+            return None
+        time.sleep(0.15)
+        self.proc.terminate()
+        sm, mx, reasons = [], [], set()
+        for ts, line in self.lines:
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9 or not (t0 - 0.1 <= ts <= t1 + 0.2):
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return None
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def oracle_shape(L):
+    cfg = L["cfg"]
+    return dict(batch=cfg.batch, Hq=cfg.n_q_heads, Hk=cfg.n_kv_heads, d=cfg.head_dim, alpha=cfg.window,
+                max_sent=L["max_sent"], slab_off=L["slab_off"], cap=L["cap"])
+
+
+def sub_layer(L, n_seq):
+    """The first n_seq sequences of a layer as a layer of their own (views, no arithmetic)."""
+    cfg = L["cfg"]
+    import dataclasses
+    rows = int((L["slab_off"][n_seq - 1] + L["cap"][n_seq - 1]) * cfg.n_kv_heads)
+    out = dict(L)
+    out["cfg"] = dataclasses.replace(cfg, batch=n_seq)
+    for k in ("cap", "slab_off", "sent_off", "sent_id", "n_sent", "kv_len", "q_win", "q", "hidden", "alpha", "flag", "ctx"):
+        out[k] = L[k][:n_seq]
+    out["K"], out["V"] = L["K"][:rows], L["V"][:rows]
+    return out
+
+
+def time_oracle(L, n_seq):
+    """One pass of the whole path by the CPU oracle over the first n_seq sequences; seconds per leg."""
+    import oracle
+    S = sub_layer(L, n_seq)
+    cfg = S["cfg"]
+    sh = oracle_shape(S)
+    Kb, Vb = W.bf16_bits(S["K"]), W.bf16_bits(S["V"])
+    t = [time.perf_counter()]
+    sc = oracle.score_batch(sh, Kb, W.bf16_bits(S["q_win"]), S["kv_len"], S["sent_off"], S["n_sent"],
+                            float(np.float32(0.1)), float(np.float32(0.95)), float(np.float32(1e-6)))
+    t.append(time.perf_counter())
+    sel = oracle.select_batch(sc["score"], S["sent_off"], S["n_sent"], cfg.budget, cfg.window)
+    t.append(time.perf_counter())
+    cp = oracle.compact_batch(sh, Kb, Vb, sel["keep"], S["sent_off"], S["sent_id"], S["n_sent"], S["kv_len"])
+    t.append(time.perf_counter())
+    oracle.decode_attn_batch(sh, W.bf16_bits(S["q"]), cp["K"], cp["V"], cp["kv_len"])
+    oracle.steer(W.bf16_bits(S["hidden"]), W.bf16_bits(S["steer_vec"]), S["alpha"], S["flag"])
+    t.append(time.perf_counter())
+    legs = dict(zip(("score", "select", "compact", "decode_attn"), np.diff(t)))
+    frac = float(S["kv_len"].sum()) / float(L["kv_len"].sum())
+    return legs, frac, oracle.max_threads()
+
+
+def run_reference(args, rank):
+    """The CPU oracle as the reference arm (rank 0 only)."""
+    if rank != 0:
+        return
+    cfg = W.config(2)
+    L = W.make_layer(cfg)
+    n_seq = 1
+    times = []
+    for i in range(args.warmup + args.steps):
+        legs, frac, cores = time_oracle(L, n_seq)
+        if i >= args.warmup:
+            times.append(legs)
+    evict_us = statistics.mean((x["score"] + x["select"] + x["compact"]) for x in times) / frac * 1e6
+    dec_s = statistics.mean(x["decode_attn"] for x in times) / frac
+    step_ms = statistics.mean(sum(x.values()) for x in times) / frac * 1e3
+    sample = f"first {n_seq} of {cfg.batch} sequences ({frac:.3f} of the tokens), time scaled by token count"
+    line = {"impl": "reference", "metric": METRIC, "value": evict_us, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": step_ms, "higher_is_better": False,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": "configs[1]: " + cfg.name, "budget": cfg.budget},
+            "decode_attn_us": dec_s * 1e6,
+            "cpu_baseline": {"value": evict_us, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": evict_us, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="skipkv", choices=["skipkv", "reference"])
+    ap.add_argument("--config", type=int, default=2, help="workload index (2 = the headline configuration)")
+    ap.add_argument("--batch", type=int, default=0, help="override the number of sequences (profiling captures)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "skipkv" else args.warmup
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+
+    from paper_2512_07993_b200 import binding as B, build
+    if not os.path.exists(B.LIB_PATH):
+        build.build()
+    B.lib()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    cfg = W.config(args.config, batch=args.batch) if args.batch else W.config(args.config)
+    L = W.make_layer(cfg)
+    D = B.DeviceLayer(L)
+    pristine = {k: getattr(D, k).clone() for k in ("K", "V", "sent_off", "sent_id", "n_sent", "kv_len", "hidden")}
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+
+    def restore():
+        for k, v in pristine.items():
+            getattr(D, k).copy_(v)
+        flush.fill_(1)                      # evict whatever the restore left in L2
+
+    legs = ("score", "select", "compact", "decode_attn")
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(args.steps)]
+
+    def step(events=None):
+        rec = (lambda i: events[i].record()) if events else (lambda i: None)
+        rec(0); D.score()
+        rec(1); D.select()
+        rec(2); D.compact()
+        rec(3); D.decode_attn(steer=True)
+        rec(4)
+
+    for _ in range(args.warmup):
+        restore(); step()
+    torch.cuda.synchronize()
+    D.status()
+    if dist: dist.barrier()
+    torch.cuda.synchronize()
+    clocks = ClockSampler(local_rank); clocks.start()
+    t0 = time.time()
+    for i in range(args.steps):
+        restore(); step(ev[i])
+    torch.cuda.synchronize()
+    if dist: dist.barrier()
+    torch.cuda.synchronize()
+    t1 = time.time()
+    clk = clocks.stop(t0, t1)
+    D.status()
+
+    per = {leg: [ev[i][k].elapsed_time(ev[i][k + 1]) * 1e3 for i in range(args.steps)] for k, leg in enumerate(legs)}
+    us = {leg: statistics.mean(v) for leg, v in per.items()}
+    us_med = {leg: statistics.median(v) for leg, v in per.items()}
+    evict_us = us["score"] + us["select"] + us["compact"]
+    step_ms = sum(us.values()) / 1e3
+    if dist:
+        tt = torch.tensor([evict_us, step_ms, us["decode_attn"]], device="cuda", dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        evict_us, step_ms, dec_us_max = tt.tolist()
+    else:
+        dec_us_max = us["decode_attn"]
+
+    # algorithmic bytes from the actual lengths
+    kv0 = L["kv_len"].astype(np.int64)
+    kv1 = D.kv_len.cpu().numpy().astype(np.int64)
+    row = 2 * cfg.head_dim
+    bytes_alg = {"score": int(kv0.sum()) * row,                      # K read once
+                 "compact": int(kv1.sum()) * row * 2 * 2,            # kept K and V rows read and written
+                 "decode_attn": int(kv1.sum()) * row * 2}            # live K and V rows read once
+    peaks = measured_peaks()
+    traffic = ncu_traffic()
+    roof = {}
+    for leg in ("score", "compact", "decode_attn"):
+        gbs = bytes_alg[leg] / (us[leg] * 1e-6) / 1e9
+        roof[leg] = {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                     "frac": gbs / peaks["hbm_gbs"], "peak_source": peaks["source"], "us": us[leg],
+                     "us_median": us_med[leg], "algorithmic_bytes": bytes_alg[leg],
+                     "frac_of_nominal_8TBs": gbs / 8000.0, "traffic": traffic.get(leg)}
+    dominant = max(("score", "compact", "decode_attn"), key=lambda k: us[k])
+
+    line = {"metric": METRIC, "value": evict_us / world, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": step_ms, "higher_is_better": False, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16 storage, f32 arithmetic", "data": "synthetic",
+            "config": {"workload": f"configs[{args.config - 1}]: {cfg.name}", "batch": cfg.batch,
+                       "kv_heads": cfg.n_kv_heads, "q_heads": cfg.n_q_heads, "head_dim": cfg.head_dim,
+                       "window": cfg.window, "budget": cfg.budget, "tokens_before": int(kv0.sum() // cfg.n_kv_heads),
+                       "tokens_after": int(kv1.sum() // cfg.n_kv_heads), "layers_per_step": 1,
+                       "l2": "256 MiB flush buffer written between iterations; inputs (1 GB) exceed L2",
+                       "replicas": world},
+            "us": us, "decode_attn_us": dec_us_max, "decode_attn_gbs": bytes_alg["decode_attn"] / (dec_us_max * 1e-6) / 1e9,
+            "roofline": dict(roof[dominant], kernel=dominant), "roofline_by_step": roof,
+            "gpu_launches": sum(LAUNCHES_PER_STEP.values()) * args.steps, "clocks": clk}
+
+    # ---- end to end through the C ABI with host buffers (pinned), copies inside the timed region
+    if not args.no_e2e:
+        host_in = {k: pristine[k].cpu().pin_memory() for k in ("K", "V", "sent_off", "sent_id", "n_sent", "kv_len", "hidden")}
+        host_in["q_win"] = D.q_win.cpu().pin_memory(); host_in["q"] = D.q.cpu().pin_memory()
+        outs = ("out", "kv_len", "n_sent", "sent_off", "sent_id", "hidden")
+        host_out = {k: torch.empty_like(getattr(D, k), device="cpu").pin_memory() for k in outs}
+        h2d = sum(v.numel() * v.element_size() for v in host_in.values())
+        d2h = sum(v.numel() * v.element_size() for v in host_out.values())
+        n_e2e = max(3, min(args.steps, 5))
+        e2e_t = []
+        for i in range(1 + n_e2e):
+            flush.fill_(1)
+            torch.cuda.synchronize()
+            a, b_, c = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+            a.record()
+            for k, v in host_in.items():
+                getattr(D, k).copy_(v, non_blocking=True)
+            D.score(); D.select(); D.compact()
+            b_.record()
+            D.decode_attn(steer=True)
+            for k in outs:
+                host_out[k].copy_(getattr(D, k), non_blocking=True)
+            c.record()
+            torch.cuda.synchronize()
+            if i:
+                e2e_t.append((a.elapsed_time(b_) * 1e3, a.elapsed_time(c) * 1e3))
+        e2e_evict = statistics.mean(x[0] for x in e2e_t)
+        e2e_all = statistics.mean(x[1] for x in e2e_t)
+        if dist:
+            tt = torch.tensor([e2e_evict, e2e_all], device="cuda", dtype=torch.float64)
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+            e2e_evict, e2e_all = tt.tolist()
+        line["e2e"] = {"value": e2e_evict / world, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                       "whole_step_us": e2e_all / world,
+                       "note": "host->device copy of K, V, queries and tables from pinned memory, the four calls, "
+                               "device->host read of the attention output, hidden state and tables"}
+
+    # ---- the oracle on this machine's host cores, bounded sample (rank 0, single GPU runs only)
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        n_seq = 1
+        legs_s, frac, cores = time_oracle(L, n_seq)
+        line["cpu_baseline"] = {"value": (legs_s["score"] + legs_s["select"] + legs_s["compact"]) / frac * 1e6,
+                                "unit": UNIT, "cores": cores, "kind": "oracle",
+                                "decode_attn_us": legs_s["decode_attn"] / frac * 1e6,
+                                "sample": f"first {n_seq} of {cfg.batch} sequences ({frac:.3f} of the tokens), "
+                                          "time scaled by token count"}
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if dist:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
