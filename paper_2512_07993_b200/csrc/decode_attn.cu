@@ -3,14 +3,15 @@
 // performed by the tail of the same launch.
 //
 // The step is HBM bound: every live K and V row is read exactly once.  Design:
-//  * Work = 64-row tiles enumerated over all (sequence, head) slabs.  The tile list is cut into
+//  * Work = 128-row tiles enumerated over all (sequence, head) slabs.  The tile list is cut into
 //    equal contiguous ranges, one per persistent CTA, so CTAs are balanced whatever the ragged
 //    lengths are; a CTA's range may cross slab boundaries, each (CTA, slab) intersection gives
 //    one partial result (running max, sum, 128-wide accumulator per head).
 //  * K and V tiles are streamed into a shared-memory ring with bulk asynchronous copies (each
 //    tile is one contiguous block of the slab) signalled through mbarriers, issued two tiles
-//    ahead by one elected lane; eight warps work on 8 rows of a tile each.  (256 threads per
-//    CTA and two CTAs per SM leave 128 registers per thread, which the mapping below needs.)
+//    ahead by one elected lane; sixteen warps work on 8 rows of a tile each.  (512 threads in one
+//    CTA per SM leave 128 registers per thread, which the mapping below needs; the ring of
+//    3 x 64 KB keeps 128 KB of loads in flight per SM.)
 //  * Consumer mapping: a half-warp per row, 8 channels (16 bytes) per lane.  The four heads of
 //    the group share every K/V load.  fp32 arithmetic with packed two-wide FMAs; the 16 partial
 //    dot products a lane holds for 4 rows x 4 heads are reduced with a 15-shuffle butterfly
@@ -24,12 +25,12 @@
 
 namespace skipkv {
 
-constexpr int kTileRows = 64;
-constexpr int kTileBytes = kTileRows * kRowBytes;         // 16 KB for K, same for V
+constexpr int kTileRows = 128;
+constexpr int kTileBytes = kTileRows * kRowBytes;         // 32 KB for K, same for V
 constexpr int kStages = 3;
-constexpr int kConsWarps = 8;
+constexpr int kConsWarps = 16;
 constexpr int kDecThreads = kConsWarps * 32;
-constexpr int kCtasPerSm = 2;
+constexpr int kCtasPerSm = 1;
 constexpr int kPartStride = 130;                          // global record: 128 accumulators + max + sum
 constexpr int kWpStride = 132;                            // same record in shared memory, 16-byte aligned rows
 constexpr int kMaxDecSlabs = 8192;
@@ -39,6 +40,18 @@ __device__ __forceinline__ float ex2(float x) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
+
+#ifdef SKIPKV_DEC_TRACE
+__device__ unsigned long long* g_dec_trace = nullptr;    // [ctas][8] nanosecond stamps (profiling builds only)
+__device__ __forceinline__ unsigned long long gtime() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+#define DEC_TRACE(slot) do { if (g_dec_trace && threadIdx.x == 0) g_dec_trace[blockIdx.x * 8 + (slot)] = gtime(); } while (0)
+#else
+#define DEC_TRACE(slot) do { } while (0)
+#endif
 
 struct DecSmem {
     uint64_t full[kStages];
@@ -151,6 +164,7 @@ decode_attn_kernel(int batch, int Hq, int Hk, int n_slabs, const int64_t* slab_o
     int* pref = reinterpret_cast<int*>(sm + 1);                              // [n_slabs + 1] tile prefix
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    DEC_TRACE(0);
     auto live = [&](int s) { return min(max(kv_len[s], 0), cap[s / Hk]); };   // live rows of slab s
     const int n = Hq / Hk;                     // heads per group
     const int NG = (n + 3) / 4;                // head groups of 4 (1 or 2)
@@ -187,6 +201,7 @@ decode_attn_kernel(int batch, int Hq, int Hk, int n_slabs, const int64_t* slab_o
         if (tid == kDecThreads - 1) pref[n_slabs] = int(run);
         __syncthreads();
     }
+    DEC_TRACE(1);
     const int Ttot = pref[n_slabs];
     const int per_cta = max(1, (Ttot + G - 1) / G);
     const int t_begin = min(cta * per_cta, Ttot), t_end = min(t_begin + per_cta, Ttot);
@@ -203,95 +218,113 @@ decode_attn_kernel(int batch, int Hq, int Hk, int n_slabs, const int64_t* slab_o
     }
 
     {
-        // ------------------------------------------------------------------ consumers
         const int hg = warp % NG;                       // head group of this warp
         const int rb = warp / NG;                       // row block: rows [rb*NG*8, (rb+1)*NG*8) of each tile
         const int half = lane >> 4, l16 = lane & 15;
         const float qscale = 1.4426950408889634f * rsqrtf(float(kHeadDim));
         float2 q2[4][4], acc[4][4];
         float m_run = -INFINITY, l_run = 0.f;
-        int slab = slab0, consumed = 0;
-        bool seg_open = false;
         bool aborted = false;
-        // copy issue (warp 0, lane 0 only): tile k of this CTA goes to stage k % kStages
+
+        // ---- copy issue (thread 0 only): the CTA's k-th tile goes to stage k % kStages.  The cursor
+        // walks the slab parts of this CTA's tile range; divisions and table reads happen once per part.
         const bool is_producer = (tid == 0);
-        int p_slab = slab0, issued = 0;
+        int p_slab = slab0, p_t = t_begin, p_rows_left = 0, p_stage = 0;
+        uint32_t p_phase = 0;                           // parity of the previous use of p_stage (first lap: no wait)
+        bool p_first_lap = true;
+        const uint8_t *p_K = K, *p_V = V;
         auto issue_next = [&]() {
-            const int tt = t_begin + issued;
-            if (tt >= t_end) return;
-            while (pref[p_slab + 1] <= tt) ++p_slab;
-            const int stage = issued % kStages, use = issued / kStages;
-            if (use > 0) {
-                if (sm->abort_flag || !mbar_wait(&sm->empty[stage], uint32_t(use - 1) & 1u)) {
+            if (p_t >= t_end) return;
+            if (p_rows_left <= 0) {
+                while (pref[p_slab + 1] <= p_t) ++p_slab;
+                const int j = p_t - pref[p_slab];
+                const size_t off =
+                    (slab_row0(slab_off, cap, Hk, p_slab / Hk, p_slab % Hk) + size_t(j) * kTileRows) * kRowBytes;
+                p_K = K + off;
+                p_V = V + off;
+                p_rows_left = live(p_slab) - j * kTileRows;
+            }
+            if (!p_first_lap) {
+                if (sm->abort_flag || !mbar_wait(&sm->empty[p_stage], p_phase)) {
                     if (!sm->abort_flag) atomicOr(status, SKIPKV_STATUS_COPY_TIMEOUT);
                     sm->abort_flag = 1;
                     return;
                 }
             }
-            const int pb = p_slab / Hk, ph = p_slab % Hk;
-            const int j = tt - pref[p_slab];
-            const int rows = min(kTileRows, live(p_slab) - j * kTileRows);
-            const size_t off = (slab_row0(slab_off, cap, Hk, pb, ph) + size_t(j) * kTileRows) * kRowBytes;
-            const uint32_t bytes = uint32_t(rows) * kRowBytes;
-            uint8_t* dstK = ring + size_t(stage) * 2 * kTileBytes;
-            mbar_expect_tx(&sm->full[stage], 2 * bytes);
-            bulk_g2s(dstK, K + off, bytes, &sm->full[stage]);
-            bulk_g2s(dstK + kTileBytes, V + off, bytes, &sm->full[stage]);
-            ++issued;
+            const uint32_t bytes = uint32_t(min(kTileRows, p_rows_left)) * kRowBytes;
+            uint8_t* dstK = ring + size_t(p_stage) * 2 * kTileBytes;
+            mbar_expect_tx(&sm->full[p_stage], 2 * bytes);
+            bulk_g2s(dstK, p_K, bytes, &sm->full[p_stage]);
+            bulk_g2s(dstK + kTileBytes, p_V, bytes, &sm->full[p_stage]);
+            p_K += kTileBytes;
+            p_V += kTileBytes;
+            p_rows_left -= kTileRows;
+            ++p_t;
+            if (++p_stage == kStages) {
+                p_stage = 0;
+                if (p_first_lap) p_first_lap = false; else p_phase ^= 1u;
+            }
         };
         if (is_producer)
             for (int k = 0; k < kStages - 1; ++k) issue_next();
-        for (int t = t_begin; t < t_end; ++t, ++consumed) {
-            if (is_producer && !sm->abort_flag) issue_next();       // keeps kStages-1 tiles in flight
+        DEC_TRACE(2);
+        bool first_tile = true;
+
+        int slab = slab0, t = t_begin, c_stage = 0;
+        uint32_t c_phase = 0;
+        while (t < t_end) {
+            // ---------------------------------------------------------- one (CTA, slab) segment
             while (pref[slab + 1] <= t) ++slab;
+            const int seg_end = min(t_end, pref[slab + 1]);
             const int b = slab / Hk, h = slab % Hk;
-            if (!seg_open) {
-                // new (CTA, slab) segment: load the group's queries, reset the running state
+            int rows_left = live(slab) - (t - pref[slab]) * kTileRows;
 #pragma unroll
-                for (int hh = 0; hh < 4; ++hh) {
-                    const int hl = hg * 4 + hh;
-                    uint4 qq = make_uint4(0u, 0u, 0u, 0u);
-                    if (hl < n)
-                        qq = reinterpret_cast<const uint4*>(q + (size_t(b) * Hq + size_t(h) * n + hl) * kHeadDim)[l16];
-                    const float2 s2 = make_float2(qscale, qscale);
-                    q2[hh][0] = __fmul2_rn(bf16x2_to_f2(qq.x), s2);
-                    q2[hh][1] = __fmul2_rn(bf16x2_to_f2(qq.y), s2);
-                    q2[hh][2] = __fmul2_rn(bf16x2_to_f2(qq.z), s2);
-                    q2[hh][3] = __fmul2_rn(bf16x2_to_f2(qq.w), s2);
+            for (int hh = 0; hh < 4; ++hh) {
+                const int hl = hg * 4 + hh;
+                uint4 qq = make_uint4(0u, 0u, 0u, 0u);
+                if (hl < n)
+                    qq = reinterpret_cast<const uint4*>(q + (size_t(b) * Hq + size_t(h) * n + hl) * kHeadDim)[l16];
+                const float2 s2 = make_float2(qscale, qscale);
+                q2[hh][0] = __fmul2_rn(bf16x2_to_f2(qq.x), s2);
+                q2[hh][1] = __fmul2_rn(bf16x2_to_f2(qq.y), s2);
+                q2[hh][2] = __fmul2_rn(bf16x2_to_f2(qq.z), s2);
+                q2[hh][3] = __fmul2_rn(bf16x2_to_f2(qq.w), s2);
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) acc[hh][c] = make_float2(0.f, 0.f);
-                }
-                m_run = -INFINITY;
-                l_run = 0.f;
-                seg_open = true;
+                for (int c = 0; c < 4; ++c) acc[hh][c] = make_float2(0.f, 0.f);
             }
-            const int stage = consumed % kStages, use = consumed / kStages;
-            const int j = t - pref[slab];
-            const int rows = min(kTileRows, live(slab) - j * kTileRows);
-            if (!aborted) {
-                if (sm->abort_flag || !mbar_wait(&sm->full[stage], uint32_t(use) & 1u)) {
-                    if (!sm->abort_flag) atomicOr(status, SKIPKV_STATUS_COPY_TIMEOUT);
-                    sm->abort_flag = 1;
-                    aborted = true;
+            m_run = -INFINITY;
+            l_run = 0.f;
+            for (; t < seg_end; ++t, rows_left -= kTileRows) {
+                if (is_producer) issue_next();                  // keeps kStages-1 tiles in flight
+                if (!aborted) {
+                    if (!mbar_wait(&sm->full[c_stage], c_phase) || sm->abort_flag) {
+                        if (!sm->abort_flag) atomicOr(status, SKIPKV_STATUS_COPY_TIMEOUT);
+                        sm->abort_flag = 1;
+                        aborted = true;
+                    }
                 }
-            }
-            if (!aborted) {
-                const uint8_t* Ks = ring + size_t(stage) * 2 * kTileBytes;
-                const uint8_t* Vs = Ks + kTileBytes;
-                for (int sub = 0; sub < NG; ++sub) {
-                    const int row_base = (rb * NG + sub) * 8;
-                    if (row_base >= rows) break;
-                    if (rows == kTileRows) tile_rows<false>(Ks, Vs, row_base, rows, lane, q2, acc, m_run, l_run);
-                    else tile_rows<true>(Ks, Vs, row_base, rows, lane, q2, acc, m_run, l_run);
+                if (first_tile) { DEC_TRACE(3); first_tile = false; }
+                if (!aborted) {
+                    const uint8_t* Ks = ring + size_t(c_stage) * 2 * kTileBytes;
+                    const uint8_t* Vs = Ks + kTileBytes;
+                    if (rows_left >= kTileRows) {
+                        for (int sub = 0; sub < NG; ++sub)
+                            tile_rows<false>(Ks, Vs, (rb * NG + sub) * 8, kTileRows, lane, q2, acc, m_run, l_run);
+                    } else {
+                        for (int sub = 0; sub < NG; ++sub) {
+                            const int row_base = (rb * NG + sub) * 8;
+                            if (row_base >= rows_left) break;
+                            tile_rows<true>(Ks, Vs, row_base, rows_left, lane, q2, acc, m_run, l_run);
+                        }
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&sm->empty[c_stage]);
                 }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&sm->empty[stage]);
+                if (++c_stage == kStages) { c_stage = 0; c_phase ^= 1u; }
             }
-            const bool seg_end = (t + 1 == t_end) || (pref[slab + 1] <= t + 1);
-            if (!seg_end) continue;
 
             // ---------------------------------------------------------- flush this (CTA, slab) segment
-            seg_open = false;
+            if (t >= t_end) DEC_TRACE(4);
             // halves of the warp hold different rows: add them; finish the sum of p
 #pragma unroll
             for (int hh = 0; hh < 4; ++hh)
@@ -372,9 +405,10 @@ decode_attn_kernel(int batch, int Hq, int Hk, int n_slabs, const int64_t* slab_o
             }
             consumer_bar();                                // wpart and is_last reusable
         }
-        // drain (only after an abort can copies still be in flight): they must land before exit
-        if (is_producer)
-            for (int k = consumed; k < issued; ++k) mbar_wait(&sm->full[k % kStages], uint32_t(k / kStages) & 1u);
+        DEC_TRACE(5);
+        // after an abort copies may still be in flight: they must land before the CTA retires
+        if (is_producer && sm->abort_flag)
+            for (int st = 0; st < kStages; ++st) { mbar_wait(&sm->full[st], 0u, 1u << 16); mbar_wait(&sm->full[st], 1u, 1u << 16); }
         // slabs with no live row: zeros (owned round-robin)
         for (int s = cta; s < n_slabs; s += G) {
             if (live(s) > 0) continue;
@@ -389,11 +423,25 @@ decode_attn_kernel(int batch, int Hq, int Hk, int n_slabs, const int64_t* slab_o
         for (int i = cta * kDecThreads + tid; i < total; i += G * kDecThreads)
             steer_vec8(i, vec_per_row, hidden, steer_vec, alpha, flag);
     }
+    DEC_TRACE(6);
+#ifdef SKIPKV_DEC_TRACE
+    if (g_dec_trace && threadIdx.x == 0) {
+        unsigned smid;
+        asm volatile("mov.u32 %0, %smid;" : "=r"(smid));
+        g_dec_trace[blockIdx.x * 8 + 7] = smid;
+    }
+#endif
 }
 
 }  // namespace skipkv
 
 using namespace skipkv;
+
+#ifdef SKIPKV_DEC_TRACE
+extern "C" int skipkv_debug_set_trace(unsigned long long* p) {
+    return cudaMemcpyToSymbol(g_dec_trace, &p, sizeof(p)) == cudaSuccess ? 0 : -4;
+}
+#endif
 
 extern "C" int skipkv_decode_attn(const skipkv_shape* shape, const void* q, const void* K, const void* V,
                                   const int32_t* kv_len, void* out, void* hidden, const void* steer_vec,
