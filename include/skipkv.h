@@ -177,6 +177,35 @@ int skipkv_steer(int32_t batch, int32_t d_model, void* hidden, const void* steer
 int skipkv_append(const skipkv_shape* shape, void* K, void* V, const void* k_new, const void* v_new,
                   int32_t* kv_len, void* ws, void* stream);
 
+/*
+ * skipkv_decode_attn_static -- skipkv_decode_attn for callers that cannot allocate device
+ * memory and so have no workspace to pass.  (The paper has no counterpart: this is a packaging
+ * variant of the same operation, not another step of the method.)  Typical callers: a serving
+ * process whose start-up gave all free HBM to the KV-cache pool, so that any later cudaMalloc
+ * fails; or an extension that must not call cudaMalloc because that call synchronises the whole
+ * device and stalls the process's other streams.  The kernel's scratch (partial results and
+ * arrival counters) lives in a fixed array inside the library instead, about 2 MB, which each
+ * GPU that loads the library holds until the process exits.  This function calls no cudaMalloc,
+ * cudaFree or other allocating routine.
+ *
+ * Arguments as skipkv_decode_attn, except that there is no workspace and that `status` (device,
+ * one uint32, nullable, caller-owned) receives the SKIPKV_STATUS_* bits by bitwise OR; the caller
+ * clears it.  Limits: batch * n_kv_heads <= SKIPKV_STATIC_MAX_SLABS, otherwise
+ * SKIPKV_ERR_UNSUPPORTED is returned, nothing is enqueued, and skipkv_last_cuda_error() says
+ * which limit was exceeded.
+ *
+ * The first call on a device looks up the array's device address and sets a kernel attribute
+ * (with that device current); make that first call before any stream capture begins.  Every call
+ * on a device shares the one array: each call first clears the counters it needs at zero (on
+ * `stream`), and two calls whose GPU work overlaps (different streams, or different threads
+ * without ordering between them) race on it and give undefined results.  Calls that follow one
+ * another on one stream are safe.
+ */
+#define SKIPKV_STATIC_MAX_SLABS 256
+int skipkv_decode_attn_static(const skipkv_shape* shape, const void* q, const void* K, const void* V,
+                              const int32_t* kv_len, void* out, void* hidden, const void* steer_vec,
+                              const float* alpha, const uint8_t* flag, uint32_t* status, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -21,7 +21,7 @@ ERRORS = {-1: "SKIPKV_ERR_INVALID_ARG", -2: "SKIPKV_ERR_UNSUPPORTED", -3: "SKIPK
           -4: "SKIPKV_ERR_CUDA", -5: "SKIPKV_ERR_TIMEOUT"}
 SYMBOLS = ["skipkv_workspace_bytes", "skipkv_workspace_init", "skipkv_status", "skipkv_last_cuda_error",
            "skipkv_score", "skipkv_select", "skipkv_compact", "skipkv_decode_attn", "skipkv_steer",
-           "skipkv_append"]
+           "skipkv_append", "skipkv_decode_attn_static"]
 
 
 class SkipKVError(RuntimeError):
@@ -74,7 +74,7 @@ def _stream(stream) -> C.c_void_p:
 
 def _check(rc: int, where: str):
     if rc != 0:
-        detail = lib().skipkv_last_cuda_error().decode() if rc == -4 else ""
+        detail = lib().skipkv_last_cuda_error().decode() if rc in (-4, -2) else ""
         raise SkipKVError(rc, where, detail)
 
 
@@ -151,6 +151,20 @@ def skipkv_append(shape, K, V, k_new, v_new, kv_len, ws, stream=None) -> None:
     _check(lib().skipkv_append(C.byref(shape), _ptr(K, torch.bfloat16), _ptr(V, torch.bfloat16),
                                _ptr(k_new, torch.bfloat16), _ptr(v_new, torch.bfloat16), _ptr(kv_len, torch.int32),
                                _ptr(ws), _stream(stream)), "skipkv_append")
+
+
+def skipkv_decode_attn_static(shape, q, K, V, kv_len, out, hidden, steer_vec, alpha, flag, status=None,
+                              stream=None) -> None:
+    """Decode attention without a workspace: scratch is a fixed array inside the library.
+
+    For callers that cannot allocate device memory.  ``status`` is an optional one-element
+    uint32-sized (int32) device tensor that receives the status bits."""
+    _check(lib().skipkv_decode_attn_static(C.byref(shape), _ptr(q, torch.bfloat16), _ptr(K, torch.bfloat16),
+                                           _ptr(V, torch.bfloat16), _ptr(kv_len, torch.int32),
+                                           _ptr(out, torch.bfloat16), _ptr(hidden, torch.bfloat16),
+                                           _ptr(steer_vec, torch.bfloat16), _ptr(alpha, torch.float32),
+                                           _ptr(flag, torch.uint8), _ptr(status, torch.int32), _stream(stream)),
+           "skipkv_decode_attn_static")
 
 
 class DeviceLayer:

@@ -13,6 +13,8 @@ int cuda_fail(cudaError_t e) {
     return SKIPKV_ERR_CUDA;
 }
 
+void set_error_text(const char* msg) { std::snprintf(g_err, sizeof(g_err), "%s", msg); }
+
 int num_sms() {
     static thread_local int cached_dev = -1, cached = 0;
     int dev = 0;

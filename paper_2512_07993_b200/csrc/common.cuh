@@ -77,6 +77,7 @@ inline WsLayout make_layout(const skipkv_shape& s) {
 
 int check_shape(const skipkv_shape* s);          // SKIPKV_OK or an error code
 int cuda_fail(cudaError_t e);                    // records the message, returns SKIPKV_ERR_CUDA
+void set_error_text(const char* msg);            // text returned by skipkv_last_cuda_error
 int num_sms();
 
 #define SKIPKV_CUDA(expr)                                            \

@@ -20,6 +20,9 @@
 //  * The last CTA to deliver a partial for a slab (self-resetting counter in the workspace)
 //    merges that slab's partials and writes the bf16 output.
 //  * Every wait is bounded; on expiry the status word is flagged and the kernel drains.
+#include <cstdio>
+#include <mutex>
+
 #include "common.cuh"
 #include "steer.cuh"
 
@@ -471,6 +474,103 @@ extern "C" int skipkv_decode_attn(const skipkv_shape* shape, const void* q, cons
         static_cast<__nv_bfloat16*>(out), &reinterpret_cast<Header*>(w + L.header)->status,
         reinterpret_cast<uint32_t*>(w + L.dec_cnt), reinterpret_cast<float*>(w + L.dec_part), shape->d_model,
         static_cast<__nv_bfloat16*>(hidden), static_cast<const __nv_bfloat16*>(steer_vec), alpha, flag);
+    SKIPKV_CUDA(cudaGetLastError());
+    return SKIPKV_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Decode attention for callers that cannot provide a workspace.
+//
+// Some callers have no device allocator to draw scratch from: a serving process that handed every
+// free byte of HBM to its KV-cache pool at start-up (so a later cudaMalloc would fail), or a
+// plug-in that is forbidden to allocate because cudaMalloc synchronises the whole device and would
+// stall the other streams of the process.  For them the partial results and arrival counters of
+// the kernel live in the fixed array below, which every GPU that loads this library holds until
+// the process exits (about 2 MB).  Sizes are therefore capped: at most SKIPKV_STATIC_MAX_SLABS
+// (sequence, head) slabs and a decode grid of at most kStaticMaxCtas CTAs.
+//
+// The array's name is only a host-side handle in host code; the device address is looked up once
+// per device with cudaGetSymbolAddress (with that device current) and handed to the kernel.
+// ---------------------------------------------------------------------------------------------
+namespace skipkv {
+
+constexpr int kStaticMaxSlabs = SKIPKV_STATIC_MAX_SLABS;
+constexpr int kStaticMaxCtas = 256;
+constexpr size_t kStaticCntOff = 256;                                      // after the status word
+constexpr size_t kStaticPartOff = kStaticCntOff + size_t(kStaticMaxSlabs) * 4;
+constexpr size_t kStaticBytes =
+    kStaticPartOff + size_t(kStaticMaxCtas + kStaticMaxSlabs) * kMaxGroup * kPartStride * 4;
+
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticBytes];
+
+constexpr int kMaxDevices = 64;
+static unsigned char* g_static_addr[kMaxDevices];      // device address of the array, per device
+static bool g_static_ready[kMaxDevices];
+static std::mutex g_static_mutex;
+
+// First call on a device: resolve the array's device address and raise the kernel's dynamic
+// shared-memory limit.  Later calls only read the cached pointer.
+static int static_setup(int dev, unsigned char** base) {
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_ready[dev]) {
+        void* p = nullptr;
+        SKIPKV_CUDA(cudaGetSymbolAddress(&p, g_static_scratch));
+        if (!p) return SKIPKV_ERR_CUDA;
+        // the device's opt-in maximum: never below what any other caller of the kernel asked for
+        int optin = 0;
+        SKIPKV_CUDA(cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
+        SKIPKV_CUDA(cudaFuncSetAttribute(decode_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, optin));
+        g_static_addr[dev] = static_cast<unsigned char*>(p);
+        g_static_ready[dev] = true;
+    }
+    *base = g_static_addr[dev];
+    return SKIPKV_OK;
+}
+
+}  // namespace skipkv
+
+extern "C" int skipkv_decode_attn_static(const skipkv_shape* shape, const void* q, const void* K, const void* V,
+                                         const int32_t* kv_len, void* out, void* hidden, const void* steer_vec,
+                                         const float* alpha, const uint8_t* flag, uint32_t* status, void* stream) {
+    if (int rc = check_shape(shape)) return rc;
+    if (!q || !K || !V || !kv_len || !out) return SKIPKV_ERR_INVALID_ARG;
+    if (hidden && (!steer_vec || !alpha || !flag || shape->d_model <= 0)) return SKIPKV_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(K) & 15) || (reinterpret_cast<uintptr_t>(V) & 15) ||
+        (reinterpret_cast<uintptr_t>(q) & 15))
+        return SKIPKV_ERR_INVALID_ARG;
+    const int slabs = shape->batch * shape->n_kv_heads;
+    if (slabs > kStaticMaxSlabs) {
+        char msg[160];
+        std::snprintf(msg, sizeof(msg),
+                      "skipkv_decode_attn_static: batch*n_kv_heads = %d exceeds SKIPKV_STATIC_MAX_SLABS = %d; "
+                      "use skipkv_decode_attn with a workspace",
+                      slabs, kStaticMaxSlabs);
+        set_error_text(msg);
+        return SKIPKV_ERR_UNSUPPORTED;
+    }
+    int dev = 0;
+    SKIPKV_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) {
+        set_error_text("skipkv_decode_attn_static: device ordinal beyond 63");
+        return SKIPKV_ERR_UNSUPPORTED;
+    }
+    const size_t smem = size_t(kStages) * 2 * kTileBytes + size_t(kConsWarps) * 4 * kWpStride * 4 + sizeof(DecSmem) +
+                        size_t(slabs + 1) * 4;
+    unsigned char* base = nullptr;
+    if (int rc = static_setup(dev, &base)) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // The array keeps whatever the previous call left: the status word and the arrival counters
+    // must start at zero (the partial records are fully written before they are read).
+    SKIPKV_CUDA(cudaMemsetAsync(base, 0, kStaticPartOff, st));
+    int grid = num_sms() * kCtasPerSm;
+    if (grid > kStaticMaxCtas) grid = kStaticMaxCtas;
+    uint32_t* status_word = status ? status : reinterpret_cast<uint32_t*>(base);
+    decode_attn_kernel<<<grid, kDecThreads, smem, st>>>(
+        shape->batch, shape->n_q_heads, shape->n_kv_heads, slabs, shape->slab_off, shape->cap,
+        static_cast<const __nv_bfloat16*>(q), static_cast<const uint8_t*>(K), static_cast<const uint8_t*>(V), kv_len,
+        static_cast<__nv_bfloat16*>(out), status_word, reinterpret_cast<uint32_t*>(base + kStaticCntOff),
+        reinterpret_cast<float*>(base + kStaticPartOff), shape->d_model, static_cast<__nv_bfloat16*>(hidden),
+        static_cast<const __nv_bfloat16*>(steer_vec), alpha, flag);
     SKIPKV_CUDA(cudaGetLastError());
     return SKIPKV_OK;
 }
