@@ -68,6 +68,8 @@ typedef struct {
     int32_t d_model;      /* hidden size of the steering add; multiple of 8                   */
     int32_t max_sent;     /* row stride of the sentence tables; every n_sent <= max_sent      */
     int32_t max_cap;      /* host-known upper bound of cap[b] (sizes grids and the workspace) */
+    int64_t total_rows;   /* rows (of head_dim bf16) in each of the K and V buffers, host-known:
+                             Hk * sum_b cap[b] for packed slabs; bounds the tiled copies         */
     const int64_t* slab_off; /* device [batch], in tokens                                     */
     const int32_t* cap;      /* device [batch], rows per (sequence, head)                     */
 } skipkv_shape;

@@ -33,7 +33,7 @@ class SkipKVError(RuntimeError):
 class Shape(C.Structure):
     _fields_ = [("batch", C.c_int32), ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32),
                 ("head_dim", C.c_int32), ("window", C.c_int32), ("d_model", C.c_int32),
-                ("max_sent", C.c_int32), ("max_cap", C.c_int32),
+                ("max_sent", C.c_int32), ("max_cap", C.c_int32), ("total_rows", C.c_int64),
                 ("slab_off", C.c_void_p), ("cap", C.c_void_p)]
 
 
@@ -79,8 +79,10 @@ def _check(rc: int, where: str):
 
 
 def make_shape(batch, n_q_heads, n_kv_heads, head_dim, window, d_model, max_sent, max_cap,
-               slab_off: Optional[torch.Tensor], cap: Optional[torch.Tensor]) -> Shape:
-    s = Shape(batch, n_q_heads, n_kv_heads, head_dim, window, d_model, max_sent, max_cap,
+               slab_off: Optional[torch.Tensor], cap: Optional[torch.Tensor], total_rows: Optional[int] = None) -> Shape:
+    if total_rows is None:                      # an upper bound is enough for calls that never tile K
+        total_rows = batch * n_kv_heads * max_cap
+    s = Shape(batch, n_q_heads, n_kv_heads, head_dim, window, d_model, max_sent, max_cap, total_rows,
               slab_off.data_ptr() if slab_off is not None else None,
               cap.data_ptr() if cap is not None else None)
     s._keepalive = (slab_off, cap)
@@ -194,7 +196,7 @@ class DeviceLayer:
         ms = int(layer["max_sent"])
         self.max_sent = ms
         self.shape = make_shape(cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.window, cfg.d_model,
-                                ms, int(layer["cap"].max()), self.slab_off, self.cap)
+                                ms, int(layer["cap"].max()), self.slab_off, self.cap, int(self.K.shape[0]))
         pt = cfg.window if cfg.protect_tail is None else cfg.protect_tail
         self.params = params or make_params(0.1, 0.95, 1e-6, cfg.budget, pt)
         bh = (cfg.batch, cfg.n_kv_heads)

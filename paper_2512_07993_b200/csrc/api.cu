@@ -3,17 +3,18 @@
 #include <cstring>
 
 #include "common.cuh"
+#include "tc.cuh"
 
 namespace skipkv {
 
 static thread_local char g_err[256] = "";
 
+void set_error_text(const char* msg) { std::snprintf(g_err, sizeof(g_err), "%s", msg); }
+
 int cuda_fail(cudaError_t e) {
     std::snprintf(g_err, sizeof(g_err), "%s: %s", cudaGetErrorName(e), cudaGetErrorString(e));
     return SKIPKV_ERR_CUDA;
 }
-
-void set_error_text(const char* msg) { std::snprintf(g_err, sizeof(g_err), "%s", msg); }
 
 int num_sms() {
     static thread_local int cached_dev = -1, cached = 0;
@@ -28,16 +29,69 @@ int num_sms() {
     return cached;
 }
 
+// cuTensorMapEncodeTiled is looked up through the runtime so the library does not link libcuda.
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            p = nullptr;
+        return reinterpret_cast<EncodeTiledFn>(p);
+    }();
+    return fn;
+}
+
+static int encode(CUtensorMap* out, const void* base, int rank, const cuuint64_t* dims, const cuuint64_t* strides,
+                  const cuuint32_t* box) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) {
+        set_error_text("cuTensorMapEncodeTiled is not available from this driver");
+        return SKIPKV_ERR_CUDA;
+    }
+    const cuuint32_t estr[3] = {1, 1, 1};
+    const CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, cuuint32_t(rank), const_cast<void*>(base), dims,
+                          strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                          CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        char msg[96];
+        std::snprintf(msg, sizeof(msg), "cuTensorMapEncodeTiled failed with CUresult %d", int(r));
+        set_error_text(msg);
+        return SKIPKV_ERR_CUDA;
+    }
+    return SKIPKV_OK;
+}
+
+int tmap_rows(CUtensorMap* out, const void* base, uint64_t rows, uint32_t box_rows) {
+    const cuuint64_t dims[2] = {cuuint64_t(kHeadDim), rows};
+    const cuuint64_t strides[1] = {cuuint64_t(kRowBytes)};
+    const cuuint32_t box[2] = {64, box_rows};
+    return encode(out, base, 2, dims, strides, box);
+}
+
+int tmap_qwin(CUtensorMap* out, const void* base, uint64_t heads, uint32_t window, uint32_t box_w, uint32_t box_heads) {
+    const cuuint64_t dims[3] = {cuuint64_t(kHeadDim), window, heads};
+    const cuuint64_t strides[2] = {cuuint64_t(kRowBytes), cuuint64_t(kRowBytes) * window};
+    const cuuint32_t box[3] = {64, box_w, box_heads};
+    return encode(out, base, 3, dims, strides, box);
+}
+
 int check_shape(const skipkv_shape* s) {
     if (!s) return SKIPKV_ERR_INVALID_ARG;
     if (s->batch <= 0 || s->n_q_heads <= 0 || s->n_kv_heads <= 0 || s->window <= 0 || s->max_sent < 0 ||
-        s->max_cap <= 0 || s->d_model < 0)
+        s->max_cap <= 0 || s->d_model < 0 || s->total_rows <= 0)
         return SKIPKV_ERR_INVALID_ARG;
     if (!s->slab_off || !s->cap) return SKIPKV_ERR_INVALID_ARG;
     if (s->head_dim != kHeadDim) return SKIPKV_ERR_UNSUPPORTED;
     if (s->n_q_heads % s->n_kv_heads != 0) return SKIPKV_ERR_UNSUPPORTED;
     const int group = s->n_q_heads / s->n_kv_heads;
     if (group > kMaxGroup || group * s->window > kMaxQRows) return SKIPKV_ERR_UNSUPPORTED;
+    if ((s->window + 128 / group - 1) / (128 / group) > kMaxQueryBlocks) return SKIPKV_ERR_UNSUPPORTED;
+    if (s->total_rows > int64_t(0x7fffffff) - 256) return SKIPKV_ERR_UNSUPPORTED;
     if (s->d_model % 8 != 0) return SKIPKV_ERR_UNSUPPORTED;
     if (int64_t(s->batch) * s->n_kv_heads > (1 << 20)) return SKIPKV_ERR_UNSUPPORTED;
     return SKIPKV_OK;

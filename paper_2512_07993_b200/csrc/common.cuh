@@ -33,17 +33,20 @@ struct WsLayout {
     size_t cp_run_dst;     // int32  [slabs][max_sent+1]  first destination token; [nruns] = new_len
     size_t dec_cnt;        // uint32 [slabs]              partials that arrived (self-resetting)
     size_t dec_part;       // float  [max_ctas + slabs][group][130]
-    size_t sc_part;        // float2 [slabs][sc_chunks][qrows]  (max, sum) of a chunk of logits
-    size_t sc_lse;         // float  [slabs][qrows]
+    size_t sc_part;        // float2 [(max_ctas + slabs) * 2][sc_rb * 128]  (max, sum) of a CTA's part of a slab
     size_t sc_tokimp;      // float  [slabs][max_cap]
-    size_t sc_vbar;        // float  [slabs][max_sent][128]
+    size_t sc_vsum;        // float  [slabs][max_sent][128]  per-sentence sums of key rows
+    size_t sc_vbar_hi;     // bf16   [slabs][max_sent][128]  normalised mean key, high part
+    size_t sc_vbar_lo;     // bf16   [slabs][max_sent][128]  and the rounding remainder
     size_t sc_z;           // float  [slabs][max_sent]
     size_t total;
-    int slabs, group, qrows, sc_chunks, dec_max_ctas;
+    int slabs, group, qrows, dec_max_ctas;
+    int sc_wb;             // window positions per query block: floor(128 / group)
+    int sc_rb;             // query blocks per group: ceil(window / sc_wb)
 };
 
-constexpr int kScoreChunk = 1024;     // tokens per sweep-1 CTA
-constexpr int kDecMaxCtas = 1024;     // upper bound of the decode grid
+constexpr int kDecMaxCtas = 1024;     // upper bound of the persistent grids
+constexpr int kMaxQueryBlocks = 4;
 
 inline size_t align256(size_t x) { return (x + 255) & ~size_t(255); }
 
@@ -52,8 +55,8 @@ inline WsLayout make_layout(const skipkv_shape& s) {
     L.slabs = s.batch * s.n_kv_heads;
     L.group = s.n_q_heads / s.n_kv_heads;
     L.qrows = L.group * s.window;
-    L.sc_chunks = (s.max_cap + kScoreChunk - 1) / kScoreChunk;
-    if (L.sc_chunks < 1) L.sc_chunks = 1;
+    L.sc_wb = 128 / (L.group > 0 ? L.group : 1);
+    L.sc_rb = (s.window + L.sc_wb - 1) / L.sc_wb;
     L.dec_max_ctas = kDecMaxCtas;
     size_t o = 0;
     auto take = [&](size_t bytes) { size_t r = o; o = align256(o + bytes); return r; };
@@ -66,10 +69,11 @@ inline WsLayout make_layout(const skipkv_shape& s) {
     L.cp_run_dst = take(slabs * (ms + 1) * 4);
     L.dec_cnt = take(slabs * 4);
     L.dec_part = take((size_t(L.dec_max_ctas) + slabs) * L.group * 130 * 4);
-    L.sc_part = take(slabs * L.sc_chunks * size_t(L.qrows) * 8);
-    L.sc_lse = take(slabs * size_t(L.qrows) * 4);
+    L.sc_part = take((size_t(L.dec_max_ctas) + slabs) * 2 * size_t(L.sc_rb) * 128 * 8);
     L.sc_tokimp = take(slabs * size_t(s.max_cap > 0 ? s.max_cap : 1) * 4);
-    L.sc_vbar = take(slabs * ms * kHeadDim * 4);
+    L.sc_vsum = take(slabs * ms * kHeadDim * 4);
+    L.sc_vbar_hi = take(slabs * ms * kHeadDim * 2);
+    L.sc_vbar_lo = take(slabs * ms * kHeadDim * 2);
     L.sc_z = take(slabs * ms * 4);
     L.total = o;
     return L;

@@ -1,21 +1,40 @@
 // skipkv_score: sentence scores per (sequence, KV head) slab (paper Section 4.1).
 //
-//   sweep 1   log-sum-exp of every window-query row over the slab's tokens (partial per chunk)
-//   combine   per-row log-sum-exp
+//   sweep 1   log-sum-exp of every window-query row over the slab's tokens
+//             (tensor cores: logits = Q_group x K_tile^T, one thread per query row)
 //   sweep 2   tok_imp[t] = (1/alpha) sum_w max_q 2^(s_q[w][t] - lse_q[w])   (max before exp: exp is monotone)
-//   pool      per sentence: mean tok_imp, mean key, normalisation
-//   gram x2   pairwise cosine G; pass 1: row sums Z_i = sum_{j!=i} e^{G_ij} and lam_i = max_{j>i} G_ij;
+//             (tensor cores: logits = K_tile x Q_group^T, one thread per token), and in the same pass
+//             the per-sentence sums of the key rows, taken from the tile already in shared memory
+//   pool      per sentence: mean tok_imp, mean key, normalisation, split into bf16 high and low parts
+//   gram x2   pairwise cosine G on the tensor cores (three bf16 products: hi.hi + hi.lo + lo.hi);
+//             pass 1: Z_i = sum_{j!=i} e^{G_ij} and lam_i = max_{j>i} G_ij;
 //             pass 2: red_i = (1/S) sum_{j!=i} e^{G_ij} / Z_j (G symmetric) and the final score.
 //
 // Logits are kept in base 2: s = (q.k) * log2(e)/sqrt(d).  |G| <= 1 so the row softmax of G
 // needs no max subtraction.
+//
+// Both sweeps are persistent, warp-specialised kernels, one CTA per SM: a TMA warp streams
+// 128-token key tiles (and the group's query block) into shared memory, one thread issues
+// tcgen05.mma into a ring of four tensor-memory accumulators, two warpgroups of epilogue warps
+// alternate over the tiles, and (sweep 2) one more warpgroup pools the key rows.  Work is the list of
+// 128-token tiles over all slabs cut into equal contiguous ranges, so ragged slabs balance.
+//
+// Query rows of a group are staged as blocks of WB = floor(128/n) window positions x n heads
+// (row q*WB + w of a block), so that the n heads of a window position sit at a fixed column
+// stride for the max over heads.
+#include <cstddef>
+
 #include "common.cuh"
+#include "tc.cuh"
 
 namespace skipkv {
 
-constexpr int kS1Tile = 32;         // tokens per shared-memory tile in sweep 1
-constexpr int kS2Tokens = 128;      // tokens (threads) per CTA in sweep 2
-constexpr int kS2RowBlk = 64;       // query rows staged per pass in sweep 2 (multiple of the group size is enforced below)
+constexpr int kAccBufs = 4;             // tensor-memory accumulators of 128 columns
+constexpr int kMaxRB = 4;               // query blocks per group
+constexpr int kSwMaxStages = 6;
+constexpr int kSw1Threads = 10 * 32;    // TMA, MMA, 8 epilogue warps
+constexpr int kSw2Threads = 14 * 32;    // + 4 pooling warps
+constexpr float kLog2e = 1.4426950408889634f;
 
 __device__ __forceinline__ float ex2f(float x) {
     float y;
@@ -23,272 +42,649 @@ __device__ __forceinline__ float ex2f(float x) {
     return y;
 }
 
-struct SlabView {
-    const uint8_t* K;      // first row of the slab
-    int N;                 // live rows
-    int b, h;
+struct SweepCtl {                       // barriers and small shared state, after the tile buffers
+    uint64_t full[kSwMaxStages], empty[kSwMaxStages];
+    uint64_t qfull, qempty;
+    uint64_t tfull[kAccBufs], tempty[kAccBufs];
+    uint32_t tmem_base;
+    int abort_flag;
+    uint32_t wsum[16];
+    alignas(16) float neg_lse[2][kMaxRB * 128];   // sweep 2: one copy per epilogue warpgroup (read as float4)
+};
+static_assert(offsetof(SweepCtl, neg_lse) % 16 == 0, "neg_lse is read with 16-byte loads");
+
+struct SweepArgs {
+    int Hq, Hk, window, n_slabs, max_cap, max_sent, RB, WB, stages;
+    const int64_t* slab_off;
+    const int32_t* cap;
+    const int32_t* kv_len;
+    const int32_t* sent_off;
+    const int32_t* n_sent;
+    float2* sc_part;                    // [(cta + slab) * 2 + warpgroup][RB * 128] (max, sum)
+    float* tok_imp_user;
+    float* tok_imp_ws;
+    float* vsum;                        // [slabs][max_sent][128] sums of key rows
+    uint32_t* status;
 };
 
-__device__ __forceinline__ SlabView slab_view(const uint8_t* K, const int64_t* slab_off, const int32_t* cap,
-                                              const int32_t* kv_len, int Hk, int slab) {
-    SlabView v;
-    v.b = slab / Hk;
-    v.h = slab % Hk;
-    v.K = K + slab_row0(slab_off, cap, Hk, v.b, v.h) * kRowBytes;
-    v.N = min(max(kv_len[slab], 0), cap[v.b]);
-    return v;
+// Bounded wait that also gives up when another role of the CTA has flagged a failure.
+__device__ __forceinline__ bool ctl_wait(SweepCtl* ctl, uint64_t* bar, uint32_t parity, uint32_t* status) {
+    if (mbar_try_wait(bar, parity)) return true;
+    for (uint32_t i = 0; i < (1u << 22); ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (i > 64) {
+            __nanosleep(64);
+            if ((i & 255) == 0 && *reinterpret_cast<volatile int*>(&ctl->abort_flag)) return false;
+        }
+    }
+    atomicOr(status, SKIPKV_STATUS_COPY_TIMEOUT);
+    *reinterpret_cast<volatile int*>(&ctl->abort_flag) = 1;
+    return false;
 }
 
-// query row r of a group (r = q_local * window + w) as 128 fp32 registers, pre-scaled
-__device__ __forceinline__ void load_row_scaled(const uint8_t* row, float scale, float (&x)[kHeadDim]) {
-    const uint4* p = reinterpret_cast<const uint4*>(row);
+// ---- sweep 1 epilogue: one accumulator (128 tokens) folded into the running (max, sum) of a row
+template <bool kMasked>
+__device__ __forceinline__ void lse_fold(uint32_t taddr, int valid, float scale, float& m, float& l) {
 #pragma unroll
-    for (int i = 0; i < 16; ++i) {
-        const uint4 u = p[i];
-        x[8 * i + 0] = bf16lo(u.x) * scale; x[8 * i + 1] = bf16hi(u.x) * scale;
-        x[8 * i + 2] = bf16lo(u.y) * scale; x[8 * i + 3] = bf16hi(u.y) * scale;
-        x[8 * i + 4] = bf16lo(u.z) * scale; x[8 * i + 5] = bf16hi(u.z) * scale;
-        x[8 * i + 6] = bf16lo(u.w) * scale; x[8 * i + 7] = bf16hi(u.w) * scale;
-    }
-}
-
-// ---------------------------------------------------------------------------------------
-// sweep 1: thread = query row (held in registers), tokens broadcast from shared memory
-// grid (chunks, slabs, row blocks of 256)
-// ---------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256)
-score_sweep1_kernel(int Hq, int Hk, int window, int qrows, int sc_chunks, const int64_t* slab_off, const int32_t* cap,
-                    const uint8_t* K, const uint8_t* q_win, const int32_t* kv_len, float2* sc_part) {
-    __shared__ __align__(16) float kt[kS1Tile][kHeadDim];
-    const int slab = blockIdx.y, chunk = blockIdx.x;
-    const SlabView sv = slab_view(K, slab_off, cap, kv_len, Hk, slab);
-    const int t0 = chunk * kScoreChunk, t1 = min(t0 + kScoreChunk, sv.N);
-    if (t0 >= sv.N) return;
-    const int n = Hq / Hk;
-    const int r = blockIdx.z * 256 + threadIdx.x;
-    const bool active = r < qrows;
-    float qv[kHeadDim];
-    if (active) {
-        // q_win[b][Hq][window][128]; rows of the group are contiguous: r = q_local*window + w
-        const uint8_t* qrow = q_win + ((size_t(sv.b) * Hq + size_t(sv.h) * n) * window + r) * kRowBytes;
-        load_row_scaled(qrow, 1.4426950408889634f * rsqrtf(float(kHeadDim)), qv);
-    }
-    float m = -INFINITY, sum = 0.f;
-    for (int tb = t0; tb < t1; tb += kS1Tile) {
-        const int nt = min(kS1Tile, t1 - tb);
-        __syncthreads();
-        // stage nt rows as fp32: 16-byte chunks, 16 per row
-        for (int i = threadIdx.x; i < nt * 16; i += blockDim.x) {
-            const int row = i >> 4, c = i & 15;
-            const uint4 u = reinterpret_cast<const uint4*>(sv.K + size_t(tb + row) * kRowBytes)[c];
-            float4* d = reinterpret_cast<float4*>(&kt[row][c * 8]);
-            d[0] = make_float4(bf16lo(u.x), bf16hi(u.x), bf16lo(u.y), bf16hi(u.y));
-            d[1] = make_float4(bf16lo(u.z), bf16hi(u.z), bf16lo(u.w), bf16hi(u.w));
-        }
-        __syncthreads();
-        if (active) {
-            for (int t = 0; t < nt; ++t) {
-                float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-                const float4* kr = reinterpret_cast<const float4*>(kt[t]);
+    for (int ch = 0; ch < 4; ++ch) {
+        if (kMasked && ch * 32 >= valid) break;
+        float v[32];
+        tmem_ld32(taddr + ch * 32, v);
+        if (kMasked) {
 #pragma unroll
-                for (int c = 0; c < 32; ++c) {
-                    const float4 k4 = kr[c];
-                    a0 = fmaf(qv[4 * c + 0], k4.x, a0);
-                    a1 = fmaf(qv[4 * c + 1], k4.y, a1);
-                    a2 = fmaf(qv[4 * c + 2], k4.z, a2);
-                    a3 = fmaf(qv[4 * c + 3], k4.w, a3);
-                }
-                const float s = (a0 + a1) + (a2 + a3);
-                if (s > m) { sum *= ex2f(m - s); m = s; }
-                sum += ex2f(s - m);
-            }
+            for (int j = 0; j < 32; ++j)
+                if (ch * 32 + j >= valid) v[j] = -INFINITY;
         }
-    }
-    if (active) sc_part[(size_t(slab) * sc_chunks + chunk) * qrows + r] = make_float2(m, sum);
-}
-
-__global__ void score_lse_kernel(int qrows, int sc_chunks, const int32_t* kv_len, const float2* sc_part,
-                                 float* sc_lse) {
-    const int slab = blockIdx.x;
-    const int N = max(kv_len[slab], 0);
-    const int nch = min(sc_chunks, (N + kScoreChunk - 1) / kScoreChunk);
-    for (int r = threadIdx.x; r < qrows; r += blockDim.x) {
-        float M = -INFINITY;
-        for (int c = 0; c < nch; ++c) M = fmaxf(M, sc_part[(size_t(slab) * sc_chunks + c) * qrows + r].x);
-        float s = 0.f;
-        for (int c = 0; c < nch; ++c) {
-            const float2 p = sc_part[(size_t(slab) * sc_chunks + c) * qrows + r];
-            s += p.y * ex2f(p.x - M);
+        float c0 = fmaxf(v[0], v[1]), c1 = fmaxf(v[2], v[3]);
+#pragma unroll
+        for (int j = 4; j < 32; j += 2) { c0 = fmaxf(c0, v[j]); c1 = fmaxf(c1, v[j + 1]); }
+        const float m_new = fmaxf(m, fmaxf(c0, c1) * scale);
+        const float neg = -m_new;
+        float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+        for (int j = 0; j < 32; j += 4) {
+            s0 += ex2f(fmaf(v[j + 0], scale, neg));
+            s1 += ex2f(fmaf(v[j + 1], scale, neg));
+            s2 += ex2f(fmaf(v[j + 2], scale, neg));
+            s3 += ex2f(fmaf(v[j + 3], scale, neg));
         }
-        sc_lse[size_t(slab) * qrows + r] = (nch > 0) ? M + log2f(s) : 0.f;
+        l = l * ex2f(m - m_new) + ((s0 + s1) + (s2 + s3));      // first chunk: 2^(-inf) = 0
+        m = m_new;
     }
 }
 
-// ---------------------------------------------------------------------------------------
-// sweep 2: thread = token (key row in registers), query rows broadcast from shared memory
-// grid (ceil(max_cap/128), slabs)
-// ---------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kS2Tokens)
-score_sweep2_kernel(int Hq, int Hk, int window, int qrows, int max_cap, const int64_t* slab_off, const int32_t* cap,
-                    const uint8_t* K, const uint8_t* q_win, const int32_t* kv_len, const float* sc_lse,
-                    float* tok_imp_user, float* tok_imp_ws) {
-    __shared__ __align__(16) float qs[kS2RowBlk][kHeadDim];
-    __shared__ float lse_s[kS2RowBlk];
-    const int slab = blockIdx.y;
-    const SlabView sv = slab_view(K, slab_off, cap, kv_len, Hk, slab);
-    const int t = blockIdx.x * kS2Tokens + threadIdx.x;
-    if (blockIdx.x * kS2Tokens >= sv.N) return;
-    const bool active = t < sv.N;
-    const int n = Hq / Hk;
-    float kv[kHeadDim];
-    if (active) load_row_scaled(sv.K + size_t(t) * kRowBytes, 1.4426950408889634f * rsqrtf(float(kHeadDim)), kv);
-    const uint8_t* qbase = q_win + (size_t(sv.b) * Hq + size_t(sv.h) * n) * window * kRowBytes;
-    const float* lse = sc_lse + size_t(slab) * qrows;
-    // window rows are staged in blocks of wb rows x n heads, laid out [w][q] so a block is contiguous in w
-    const int wb = kS2RowBlk / n;
+// ---- sweep 2 epilogue: one accumulator (this thread's token x one query block) added to the token's total
+template <int kN>
+__device__ __forceinline__ float imp_fold(uint32_t taddr, const float* neg_lse, int wvalid, float scale) {
+    constexpr int WB = 128 / kN;
+    float best[WB];
     float total = 0.f;
-    for (int w0 = 0; w0 < window; w0 += wb) {
-        const int nw = min(wb, window - w0);
-        __syncthreads();
-        for (int i = threadIdx.x; i < nw * n * 16; i += kS2Tokens) {
-            const int lr = i >> 4, c = i & 15;            // local row lr = wl * n + ql
-            const int wl = lr / n, ql = lr % n;
-            const uint4 u = reinterpret_cast<const uint4*>(qbase + (size_t(ql) * window + (w0 + wl)) * kRowBytes)[c];
-            float4* d = reinterpret_cast<float4*>(&qs[lr][c * 8]);
-            d[0] = make_float4(bf16lo(u.x), bf16hi(u.x), bf16lo(u.y), bf16hi(u.y));
-            d[1] = make_float4(bf16lo(u.z), bf16hi(u.z), bf16lo(u.w), bf16hi(u.w));
-        }
-        for (int i = threadIdx.x; i < nw * n; i += kS2Tokens) {
-            const int wl = i / n, ql = i % n;
-            lse_s[i] = lse[ql * window + (w0 + wl)];
-        }
-        __syncthreads();
-        if (active) {
-            for (int wl = 0; wl < nw; ++wl) {
-                float best = -INFINITY;
-                for (int ql = 0; ql < n; ++ql) {
-                    const float4* qr = reinterpret_cast<const float4*>(qs[wl * n + ql]);
-                    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
 #pragma unroll
-                    for (int c = 0; c < 32; ++c) {
-                        const float4 q4 = qr[c];
-                        a0 = fmaf(kv[4 * c + 0], q4.x, a0);
-                        a1 = fmaf(kv[4 * c + 1], q4.y, a1);
-                        a2 = fmaf(kv[4 * c + 2], q4.z, a2);
-                        a3 = fmaf(kv[4 * c + 3], q4.w, a3);
-                    }
-                    best = fmaxf(best, ((a0 + a1) + (a2 + a3)) - lse_s[wl * n + ql]);
+    for (int ch = 0; ch < 4; ++ch) {
+        if (ch * 32 >= kN * WB) break;
+        float v[32];
+        tmem_ld32(taddr + ch * 32, v);
+#pragma unroll
+        for (int j4 = 0; j4 < 32; j4 += 4) {
+            const float4 nl = *reinterpret_cast<const float4*>(neg_lse + ch * 32 + j4);
+            const float nls[4] = {nl.x, nl.y, nl.z, nl.w};
+#pragma unroll
+            for (int jj = 0; jj < 4; ++jj) {
+                const int c = ch * 32 + j4 + jj;
+                if (c < kN * WB) {
+                    const int q = c / WB, w = c % WB;
+                    const float x = fmaf(v[j4 + jj], scale, nls[jj]);
+                    best[w] = (q == 0) ? x : fmaxf(best[w], x);
+                    if (q == kN - 1) total += (w < wvalid) ? ex2f(best[w]) : 0.f;
                 }
-                total += ex2f(best);
             }
         }
     }
-    if (active) {
-        const float v = total / float(window);
-        tok_imp_ws[size_t(slab) * max_cap + t] = v;
-        if (tok_imp_user) tok_imp_user[slab_row0(slab_off, cap, Hk, sv.b, sv.h) + t] = v;
+    return total;
+}
+
+template <int kSweep, int kN>
+__global__ void __launch_bounds__(kSweep == 1 ? kSw1Threads : kSw2Threads, 1)
+score_sweep_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapQ,
+                   const SweepArgs a) {
+    extern __shared__ uint8_t sweep_smem_raw[];
+    constexpr int kThreads = kSweep == 1 ? kSw1Threads : kSw2Threads;
+    const uint32_t raw = smem_u32(sweep_smem_raw);
+    uint8_t* tiles = sweep_smem_raw + (((raw + 1023u) & ~1023u) - raw);          // 1024-byte aligned
+    uint8_t* qbuf = tiles + size_t(a.stages) * kOpBytes;
+    SweepCtl* ctl = reinterpret_cast<SweepCtl*>(qbuf + size_t(a.RB) * kOpBytes);
+    int* pref = reinterpret_cast<int*>(ctl + 1);                                 // [n_slabs + 1] tile prefix
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int G = gridDim.x, cta = blockIdx.x;
+    const int n_slabs = a.n_slabs, Hk = a.Hk, RB = a.RB;
+    auto live = [&](int s) { return min(max(a.kv_len[s], 0), a.cap[s / Hk]); };
+
+    if (tid == 0) {
+        for (int s = 0; s < kSwMaxStages; ++s) {
+            mbar_init(&ctl->full[s], 1);
+            mbar_init(&ctl->empty[s], kSweep == 1 ? 1 : 5);      // MMA commit (+ 4 pooling warps)
+        }
+        mbar_init(&ctl->qfull, 1);
+        mbar_init(&ctl->qempty, 1);
+        for (int b = 0; b < kAccBufs; ++b) { mbar_init(&ctl->tfull[b], 1); mbar_init(&ctl->tempty[b], 4); }
+        ctl->abort_flag = 0;
+        mbar_fence_init();
+        tmap_prefetch(&mapK);
+        tmap_prefetch(&mapQ);
+    }
+    if (warp == 1) tmem_alloc(&ctl->tmem_base, 512);
+    // tile prefix over slabs (block scan; every thread owns a contiguous block of slabs)
+    {
+        const int per = (n_slabs + kThreads - 1) / kThreads;
+        const int s0 = min(tid * per, n_slabs), s1 = min(s0 + per, n_slabs);
+        uint32_t local = 0;
+        for (int s = s0; s < s1; ++s) local += uint32_t((live(s) + 127) >> 7);
+        uint32_t inc = local;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const uint32_t x = __shfl_up_sync(0xffffffffu, inc, d);
+            if (lane >= d) inc += x;
+        }
+        if (lane == 31) ctl->wsum[warp] = inc;
+        tc_fence_before();
+        __syncthreads();                                 // also publishes barrier inits and the tmem address
+        tc_fence_after();
+        uint32_t base = 0;
+        for (int w = 0; w < warp; ++w) base += ctl->wsum[w];
+        uint32_t run = base + inc - local;
+        for (int s = s0; s < s1; ++s) {
+            pref[s] = int(run);
+            run += uint32_t((live(s) + 127) >> 7);
+        }
+        if (tid == kThreads - 1) pref[n_slabs] = int(run);
+        __syncthreads();
+    }
+    const uint32_t tmem_base = ctl->tmem_base;
+    const int Ttot = pref[n_slabs];
+    const int per_cta = max(1, (Ttot + G - 1) / G);
+    const int t_begin = min(cta * per_cta, Ttot), t_end = min(t_begin + per_cta, Ttot);
+    const int ntl = t_end - t_begin;
+    int slab0 = 0;
+    if (ntl > 0) {
+        int lo = 0, hi = n_slabs - 1;
+        while (lo < hi) {
+            const int mid = (lo + hi + 1) >> 1;
+            if (pref[mid] <= t_begin) lo = mid; else hi = mid - 1;
+        }
+        slab0 = lo;
+    }
+    const float scale = kLog2e * rsqrtf(float(kHeadDim));
+    const int n = a.Hq / Hk;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0 && ntl > 0) {
+            int slab = slab0, stage = 0, issued = 0;
+            uint32_t lap = 0, qlap = 0;
+            bool ok = true;
+            for (int t = t_begin; t < t_end && ok; ++t) {
+                if (t == t_begin || pref[slab + 1] <= t) {
+                    while (pref[slab + 1] <= t) ++slab;
+                    if (qlap > 0) ok = ctl_wait(ctl, &ctl->qempty, (qlap - 1) & 1u, a.status);
+                    if (!ok) break;
+                    const int b = slab / Hk, h = slab % Hk;
+                    mbar_expect_tx(&ctl->qfull, uint32_t(RB) * 2u * 128u * uint32_t(a.WB * n));
+                    for (int k = 0; k < RB; ++k) {
+                        tma_load_3d(qbuf + size_t(k) * kOpBytes, &mapQ, 0, k * a.WB, b * a.Hq + h * n, &ctl->qfull);
+                        tma_load_3d(qbuf + size_t(k) * kOpBytes + kOpHalfBytes, &mapQ, 64, k * a.WB, b * a.Hq + h * n,
+                                    &ctl->qfull);
+                    }
+                    ++qlap;
+                }
+                if (lap > 0) ok = ctl_wait(ctl, &ctl->empty[stage], (lap - 1) & 1u, a.status);
+                if (!ok) break;
+                const long long row = (long long)slab_row0(a.slab_off, a.cap, Hk, slab / Hk, slab % Hk) +
+                                      (long long)(t - pref[slab]) * 128;
+                uint8_t* dst = tiles + size_t(stage) * kOpBytes;
+                mbar_expect_tx(&ctl->full[stage], kOpBytes);
+                tma_load_2d(dst, &mapK, 0, int(row), &ctl->full[stage]);
+                tma_load_2d(dst + kOpHalfBytes, &mapK, 64, int(row), &ctl->full[stage]);
+                ++issued;
+                if (++stage == a.stages) { stage = 0; ++lap; }
+            }
+            if (!ok) {
+                // copies already issued must land before the CTA retires
+                for (int s = 0; s < a.stages; ++s) { mbar_wait(&ctl->full[s], 0u, 1u << 16); mbar_wait(&ctl->full[s], 1u, 1u << 16); }
+                mbar_wait(&ctl->qfull, 0u, 1u << 16);
+                mbar_wait(&ctl->qfull, 1u, 1u << 16);
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0 && ntl > 0) {
+            int slab = slab0, stage = 0, it = 0;
+            uint32_t lap = 0, qlap = 0;
+            bool ok = true;
+            for (int t = t_begin; t < t_end && ok; ++t) {
+                if (t == t_begin || pref[slab + 1] <= t) {
+                    while (pref[slab + 1] <= t) ++slab;
+                    ok = ctl_wait(ctl, &ctl->qfull, qlap & 1u, a.status);
+                    if (!ok) break;
+                    ++qlap;
+                }
+                ok = ctl_wait(ctl, &ctl->full[stage], lap & 1u, a.status);
+                if (!ok) break;
+                const uint32_t k_smem = smem_u32(tiles + size_t(stage) * kOpBytes);
+                for (int k = 0; k < RB && ok; ++k, ++it) {
+                    const int buf = it & (kAccBufs - 1), use = it / kAccBufs;
+                    if (use > 0) ok = ctl_wait(ctl, &ctl->tempty[buf], uint32_t(use - 1) & 1u, a.status);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t q_smem = smem_u32(qbuf + size_t(k) * kOpBytes);
+                    if (kSweep == 1) umma_tile_128x128x128(tmem_base + buf * 128, q_smem, k_smem, false);
+                    else             umma_tile_128x128x128(tmem_base + buf * 128, k_smem, q_smem, false);
+                    umma_commit(&ctl->tfull[buf]);
+                }
+                umma_commit(&ctl->empty[stage]);
+                if (t + 1 == t_end || pref[slab + 1] <= t + 1) umma_commit(&ctl->qempty);
+                if (++stage == a.stages) { stage = 0; ++lap; }
+            }
+        }
+    } else if (warp < 10) {
+        // ------------------------------------------------------------------ epilogue warpgroups
+        const int g = (warp - 2) >> 2;                       // warpgroup: tiles t_begin + g, + g + 2, ...
+        const int quarter = warp & 3;                        // tensor-memory lanes this warp may read
+        const int row = quarter * 32 + lane;
+        const uint32_t lane_addr = tmem_base + (uint32_t(quarter * 32) << 16);
+        bool ok = true;
+        int slab = slab0, tl = g;
+        if (kSweep == 1) {
+            for (int seg_t = t_begin; seg_t < t_end;) {
+                while (pref[slab + 1] <= seg_t) ++slab;
+                const int seg_end = min(t_end, pref[slab + 1]);
+                const int N = live(slab);
+                float m[kMaxRB], l[kMaxRB];
+#pragma unroll
+                for (int k = 0; k < kMaxRB; ++k) { m[k] = -INFINITY; l[k] = 0.f; }
+                for (; t_begin + tl < seg_end; tl += 2) {
+                    const int t = t_begin + tl;
+                    const int valid = min(128, N - (t - pref[slab]) * 128);
+#pragma unroll
+                    for (int k = 0; k < kMaxRB; ++k) {
+                        if (k < RB && ok) {
+                            const int it = tl * RB + k, buf = it & (kAccBufs - 1);
+                            ok = ctl_wait(ctl, &ctl->tfull[buf], uint32_t(it / kAccBufs) & 1u, a.status);
+                            ok = __all_sync(0xffffffffu, ok);
+                            if (ok) {
+                                tc_fence_after();
+                                if (valid == 128) lse_fold<false>(lane_addr + buf * 128, valid, scale, m[k], l[k]);
+                                else              lse_fold<true>(lane_addr + buf * 128, valid, scale, m[k], l[k]);
+                                tc_fence_before();
+                                __syncwarp();
+                                if (lane == 0) mbar_arrive(&ctl->tempty[buf]);
+                            }
+                        }
+                    }
+                }
+                float2* rec = a.sc_part + (size_t(cta + slab) * 2 + g) * (size_t(RB) * 128);
+#pragma unroll
+                for (int k = 0; k < kMaxRB; ++k)
+                    if (k < RB) rec[k * 128 + row] = make_float2(m[k], l[k]);
+                seg_t = seg_end;
+            }
+        } else {
+            float* nl = ctl->neg_lse[g];
+            const int wt = tid - 64 - g * 128;              // thread index inside the warpgroup
+            int N = 0;
+            size_t row0 = 0;
+            bool have = false;
+            for (; tl < ntl; tl += 2) {
+                const int t = t_begin + tl;
+                if (!have || pref[slab + 1] <= t) {
+                    while (pref[slab + 1] <= t) ++slab;
+                    have = true;
+                    N = live(slab);
+                    row0 = slab_row0(a.slab_off, a.cap, Hk, slab / Hk, slab % Hk);
+                    // log-sum-exp of every query row of this slab from the sweep-1 records
+                    const int fc = pref[slab] / per_cta, lc = (pref[slab + 1] - 1) / per_cta;
+                    const float2* r0 = a.sc_part + size_t(fc + slab) * 2 * (size_t(RB) * 128);
+                    const int n_part = (lc - fc + 1) * 2;
+                    named_bar_sync(2 + g, 128);              // previous readers of nl are done
+                    for (int k = 0; k < RB; ++k) {
+                        float M = -INFINITY;
+                        for (int p = 0; p < n_part; ++p) M = fmaxf(M, r0[size_t(p) * RB * 128 + k * 128 + wt].x);
+                        float L = 0.f;
+                        for (int p = 0; p < n_part; ++p) {
+                            const float2 pr = r0[size_t(p) * RB * 128 + k * 128 + wt];
+                            if (pr.y > 0.f) L += pr.y * ex2f(pr.x - M);
+                        }
+                        nl[k * 128 + wt] = (L > 0.f) ? -(M + log2f(L)) : 0.f;
+                    }
+                    named_bar_sync(2 + g, 128);
+                }
+                float total = 0.f;
+#pragma unroll
+                for (int k = 0; k < kMaxRB; ++k) {
+                    if (k < RB && ok) {
+                        const int it = tl * RB + k, buf = it & (kAccBufs - 1);
+                        ok = ctl_wait(ctl, &ctl->tfull[buf], uint32_t(it / kAccBufs) & 1u, a.status);
+                        ok = __all_sync(0xffffffffu, ok);
+                        if (ok) {
+                            tc_fence_after();
+                            total += imp_fold<kN>(lane_addr + buf * 128, nl + k * 128,
+                                                  min(128 / kN, a.window - k * (128 / kN)), scale);
+                            tc_fence_before();
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(&ctl->tempty[buf]);
+                        }
+                    }
+                }
+                const int tok = (t - pref[slab]) * 128 + row;
+                if (ok && tok < N) {
+                    const float v = total / float(a.window);
+                    a.tok_imp_ws[size_t(slab) * a.max_cap + tok] = v;
+                    if (a.tok_imp_user) a.tok_imp_user[row0 + tok] = v;
+                }
+            }
+        }
+    } else if (kSweep == 2) {
+        // ------------------------------------------------------------------ pooling warps: per-sentence sums of key rows
+        const int pt = tid - 320, g2 = pt >> 6, c2 = pt & 63;          // two groups of 64 rows; 2 channels per thread
+        const int half = c2 >> 5, chunk = (c2 & 31) >> 2, within = c2 & 3;
+        int slab = slab0, S = 0, N = 0, cur = -1;
+        const int32_t* so = a.sent_off;
+        bool ok = true, have = false;
+        for (int tl = 0; tl < ntl && ok; ++tl) {
+            const int t = t_begin + tl, stage = tl % a.stages;
+            ok = ctl_wait(ctl, &ctl->full[stage], uint32_t(tl / a.stages) & 1u, a.status);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            if (!have || pref[slab + 1] <= t) {
+                while (pref[slab + 1] <= t) ++slab;
+                have = true;
+                S = min(max(a.n_sent[slab], 0), a.max_sent);
+                so = a.sent_off + size_t(slab) * (a.max_sent + 1);
+                N = live(slab);
+                cur = -1;
+            }
+            const int tok0 = (t - pref[slab]) * 128;
+            const int r_lo = g2 * 64, r_hi = min(r_lo + 64, N - tok0);
+            if (S > 0 && r_lo < r_hi) {
+                const int tk = tok0 + r_lo;
+                if (cur < 0) {
+                    int lo = 0, hi = S - 1;
+                    while (lo < hi) {
+                        const int mid = (lo + hi + 1) >> 1;
+                        if (so[mid] <= tk) lo = mid; else hi = mid - 1;
+                    }
+                    cur = lo;
+                } else {
+                    while (cur + 1 < S && so[cur + 1] <= tk) ++cur;
+                }
+                const uint8_t* colbase = tiles + size_t(stage) * kOpBytes + half * kOpHalfBytes + within * 4;
+                int r = r_lo;
+                while (r < r_hi) {
+                    int e = r_hi;
+                    if (cur + 1 < S) e = min(e, so[cur + 1] - tok0);
+                    if (e > r) {
+                        float a0 = 0.f, a1 = 0.f;
+                        for (; r < e; ++r) {
+                            const uint32_t u =
+                                *reinterpret_cast<const uint32_t*>(colbase + r * 128 + ((chunk ^ (r & 7)) << 4));
+                            a0 += bf16lo(u);
+                            a1 += bf16hi(u);
+                        }
+                        atomicAdd(reinterpret_cast<float2*>(a.vsum + (size_t(slab) * a.max_sent + cur) * kHeadDim) + c2,
+                                  make_float2(a0, a1));
+                    }
+                    if (r < r_hi) ++cur;                     // the piece ended on a sentence boundary
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&ctl->empty[stage]);
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, 512);
     }
 }
 
 // ---------------------------------------------------------------------------------------
-// pooling: one warp per sentence, 4 channels per lane
+// pooling: one warp per sentence, 4 channels per lane; writes the normalised mean key as bf16 hi + lo
 // ---------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256)
-score_pool_kernel(int Hk, int max_sent, int max_cap, const int64_t* slab_off, const int32_t* cap, const uint8_t* K,
-                  const int32_t* kv_len, const int32_t* sent_off, const int32_t* n_sent, float eps,
-                  const float* tok_imp_ws, float* sent_imp, float* sc_vbar) {
+score_pool_kernel(int Hk, int max_sent, int max_cap, const int32_t* cap, const int32_t* kv_len,
+                  const int32_t* sent_off, const int32_t* n_sent, float eps, const float* tok_imp_ws,
+                  const float* vsum, float* sent_imp, __nv_bfloat16* vbar_hi, __nv_bfloat16* vbar_lo) {
     const int slab = blockIdx.y;
     const int lane = threadIdx.x & 31;
     const int i = blockIdx.x * 8 + (threadIdx.x >> 5);
     const int S = min(n_sent[slab], max_sent);
     if (i >= S) return;
-    const SlabView sv = slab_view(K, slab_off, cap, kv_len, Hk, slab);
+    const int N = min(max(kv_len[slab], 0), cap[slab / Hk]);
     const int32_t* so = sent_off + size_t(slab) * (max_sent + 1);
-    const int b = max(so[i], 0), e = min(so[i + 1], sv.N);
-    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f, ti = 0.f;
-    for (int t = b; t < e; ++t) {
-        const uint2 u = reinterpret_cast<const uint2*>(sv.K + size_t(t) * kRowBytes)[lane];
-        a0 += bf16lo(u.x); a1 += bf16hi(u.x); a2 += bf16lo(u.y); a3 += bf16hi(u.y);
-    }
+    const int b = max(so[i], 0), e = min(so[i + 1], N);
+    float ti = 0.f;
     for (int t = b + lane; t < e; t += 32) ti += tok_imp_ws[size_t(slab) * max_cap + t];
     const float len = float(max(e - b, 1));
-    a0 /= len; a1 /= len; a2 /= len; a3 /= len;
-    float nn = a0 * a0 + a1 * a1 + a2 * a2 + a3 * a3;
+    const size_t o = (size_t(slab) * max_sent + i) * kHeadDim;
+    float4 v = reinterpret_cast<const float4*>(vsum + o)[lane];
+    if (e <= b) v = make_float4(0.f, 0.f, 0.f, 0.f);
+    v.x /= len; v.y /= len; v.z /= len; v.w /= len;
+    float nn = v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
 #pragma unroll
     for (int d = 16; d; d >>= 1) {
         nn += __shfl_xor_sync(0xffffffffu, nn, d);
         ti += __shfl_xor_sync(0xffffffffu, ti, d);
     }
     const float inv = 1.f / (sqrtf(nn) + eps);
-    reinterpret_cast<float4*>(sc_vbar + (size_t(slab) * max_sent + i) * kHeadDim)[lane] =
-        make_float4(a0 * inv, a1 * inv, a2 * inv, a3 * inv);
+    const float x[4] = {v.x * inv, v.y * inv, v.z * inv, v.w * inv};
+    uint32_t hi[4], lo[4];                                   // bf16 bit patterns
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+        const __nv_bfloat16 h = __float2bfloat16_rn(x[c]);
+        const __nv_bfloat16 r = __float2bfloat16_rn(x[c] - __bfloat162float(h));
+        hi[c] = __bfloat16_as_ushort(h);
+        lo[c] = __bfloat16_as_ushort(r);
+    }
+    reinterpret_cast<uint2*>(vbar_hi + o)[lane] = make_uint2(hi[0] | (hi[1] << 16), hi[2] | (hi[3] << 16));
+    reinterpret_cast<uint2*>(vbar_lo + o)[lane] = make_uint2(lo[0] | (lo[1] << 16), lo[2] | (lo[3] << 16));
     if (lane == 0) sent_imp[size_t(slab) * max_sent + i] = (e > b) ? ti / len : 0.f;
 }
 
 // ---------------------------------------------------------------------------------------
-// Gram passes: CTA = 32 sentences i (one per warp) x all j in tiles of 32 (one per lane)
+// Gram passes on the tensor cores.  CTA = 128 sentences i of one slab against all j in blocks of 128.
 // ---------------------------------------------------------------------------------------
-template <int kPass>
-__global__ void __launch_bounds__(1024)
-score_gram_kernel(int max_sent, const int32_t* n_sent, float sigma, float tau, const float* sc_vbar, float* sc_z,
-                  const float* sent_imp, float* sent_red, float* sent_lam, float* sent_score) {
-    __shared__ float vi[32][kHeadDim];
-    __shared__ float vj[32][kHeadDim + 1];
-    const int slab = blockIdx.y;
-    const int S = min(n_sent[slab], max_sent);
-    const int i0 = blockIdx.x * 32;
-    if (i0 >= S) return;
-    const int ti = threadIdx.x >> 5, tj = threadIdx.x & 31;
-    const int i = i0 + ti;
-    const float* vb = sc_vbar + size_t(slab) * max_sent * kHeadDim;
-    for (int k = threadIdx.x; k < 32 * kHeadDim; k += 1024) {
-        const int r = k / kHeadDim, c = k % kHeadDim;
-        vi[r][c] = (i0 + r < S) ? vb[size_t(i0 + r) * kHeadDim + c] : 0.f;
+struct GramCtl {
+    uint64_t afull, bfull[2], bempty[2], tfull[2], tempty[2];
+    uint32_t tmem_base;
+    int abort_flag;
+    float invz[2][128];
+};
+constexpr int kGramThreads = 6 * 32;
+constexpr size_t kGramSmem = 1024 + 6 * size_t(kOpBytes) + sizeof(GramCtl);
+
+__device__ __forceinline__ bool gram_wait(GramCtl* ctl, uint64_t* bar, uint32_t parity, uint32_t* status) {
+    if (mbar_try_wait(bar, parity)) return true;
+    for (uint32_t i = 0; i < (1u << 22); ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (i > 64) {
+            __nanosleep(64);
+            if ((i & 255) == 0 && *reinterpret_cast<volatile int*>(&ctl->abort_flag)) return false;
+        }
     }
-    float accum = 0.f, mx = -INFINITY;
-    for (int j0 = 0; j0 < S; j0 += 32) {
-        __syncthreads();
-        for (int k = threadIdx.x; k < 32 * kHeadDim; k += 1024) {
-            const int r = k / kHeadDim, c = k % kHeadDim;
-            vj[r][c] = (j0 + r < S) ? vb[size_t(j0 + r) * kHeadDim + c] : 0.f;
+    atomicOr(status, SKIPKV_STATUS_COPY_TIMEOUT);
+    *reinterpret_cast<volatile int*>(&ctl->abort_flag) = 1;
+    return false;
+}
+
+template <int kPass>
+__global__ void __launch_bounds__(kGramThreads, 1)
+score_gram_kernel(const __grid_constant__ CUtensorMap mapHi, const __grid_constant__ CUtensorMap mapLo, int max_sent,
+                  const int32_t* n_sent, float sigma, float tau, float* sc_z, const float* sent_imp, float* sent_red,
+                  float* sent_lam, float* sent_score, uint32_t* status) {
+    extern __shared__ uint8_t gram_smem_raw[];
+    const int slab = blockIdx.y;
+    const int S = min(max(n_sent[slab], 0), max_sent);
+    const int i0 = blockIdx.x * 128;
+    if (i0 >= S) return;
+    const uint32_t raw = smem_u32(gram_smem_raw);
+    uint8_t* At = gram_smem_raw + (((raw + 1023u) & ~1023u) - raw);              // hi, lo of the i block
+    uint8_t* Bt = At + 2 * kOpBytes;                                             // 2 stages x (hi, lo) of a j block
+    GramCtl* ctl = reinterpret_cast<GramCtl*>(Bt + 4 * kOpBytes);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int NJ = (S + 127) >> 7;
+    const int rowbase = slab * max_sent;
+
+    if (tid == 0) {
+        mbar_init(&ctl->afull, 1);
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(&ctl->bfull[s], 1);
+            mbar_init(&ctl->bempty[s], 1);
+            mbar_init(&ctl->tfull[s], 1);
+            mbar_init(&ctl->tempty[s], 4);
         }
-        __syncthreads();
-        const int j = j0 + tj;
-        float g0 = 0.f, g1 = 0.f, g2 = 0.f, g3 = 0.f;
-#pragma unroll 8
-        for (int c = 0; c < kHeadDim; c += 4) {
-            g0 = fmaf(vi[ti][c + 0], vj[tj][c + 0], g0);
-            g1 = fmaf(vi[ti][c + 1], vj[tj][c + 1], g1);
-            g2 = fmaf(vi[ti][c + 2], vj[tj][c + 2], g2);
-            g3 = fmaf(vi[ti][c + 3], vj[tj][c + 3], g3);
+        ctl->abort_flag = 0;
+        mbar_fence_init();
+        tmap_prefetch(&mapHi);
+        tmap_prefetch(&mapLo);
+    }
+    if (warp == 1) tmem_alloc(&ctl->tmem_base, 256);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = ctl->tmem_base;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            mbar_expect_tx(&ctl->afull, 2 * kOpBytes);
+            tma_load_2d(At, &mapHi, 0, rowbase + i0, &ctl->afull);
+            tma_load_2d(At + kOpHalfBytes, &mapHi, 64, rowbase + i0, &ctl->afull);
+            tma_load_2d(At + kOpBytes, &mapLo, 0, rowbase + i0, &ctl->afull);
+            tma_load_2d(At + kOpBytes + kOpHalfBytes, &mapLo, 64, rowbase + i0, &ctl->afull);
+            bool ok = true;
+            for (int jb = 0; jb < NJ && ok; ++jb) {
+                const int s = jb & 1;
+                if (jb >= 2) ok = gram_wait(ctl, &ctl->bempty[s], uint32_t((jb >> 1) - 1) & 1u, status);
+                if (!ok) break;
+                uint8_t* dst = Bt + size_t(s) * 2 * kOpBytes;
+                mbar_expect_tx(&ctl->bfull[s], 2 * kOpBytes);
+                tma_load_2d(dst, &mapHi, 0, rowbase + jb * 128, &ctl->bfull[s]);
+                tma_load_2d(dst + kOpHalfBytes, &mapHi, 64, rowbase + jb * 128, &ctl->bfull[s]);
+                tma_load_2d(dst + kOpBytes, &mapLo, 0, rowbase + jb * 128, &ctl->bfull[s]);
+                tma_load_2d(dst + kOpBytes + kOpHalfBytes, &mapLo, 64, rowbase + jb * 128, &ctl->bfull[s]);
+            }
+            if (!ok) {
+                mbar_wait(&ctl->afull, 0u, 1u << 16);
+                for (int s = 0; s < 2; ++s) { mbar_wait(&ctl->bfull[s], 0u, 1u << 16); mbar_wait(&ctl->bfull[s], 1u, 1u << 16); }
+            }
         }
-        const float g = (g0 + g1) + (g2 + g3);
-        if (j < S && j != i && i < S) {
-            const float e = __expf(g);
+    } else if (warp == 1) {
+        if (lane == 0) {
+            bool ok = gram_wait(ctl, &ctl->afull, 0u, status);
+            const uint32_t a_hi = smem_u32(At), a_lo = smem_u32(At + kOpBytes);
+            for (int jb = 0; jb < NJ && ok; ++jb) {
+                const int s = jb & 1;
+                ok = gram_wait(ctl, &ctl->bfull[s], uint32_t(jb >> 1) & 1u, status);
+                if (ok && jb >= 2) ok = gram_wait(ctl, &ctl->tempty[s], uint32_t((jb >> 1) - 1) & 1u, status);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t b_hi = smem_u32(Bt + size_t(s) * 2 * kOpBytes), b_lo = b_hi + kOpBytes;
+                const uint32_t d = tmem_base + s * 128;
+                umma_tile_128x128x128(d, a_hi, b_hi, false);
+                umma_tile_128x128x128(d, a_hi, b_lo, true);
+                umma_tile_128x128x128(d, a_lo, b_hi, true);
+                umma_commit(&ctl->tfull[s]);
+                umma_commit(&ctl->bempty[s]);
+            }
+        }
+    } else {
+        const int quarter = warp & 3, wt = tid - 64;
+        const int i = i0 + quarter * 32 + lane;
+        const uint32_t lane_addr = tmem_base + (uint32_t(quarter * 32) << 16);
+        float accum = 0.f, mx = -INFINITY;
+        bool ok = true;
+        for (int jb = 0; jb < NJ && ok; ++jb) {
+            const int s = jb & 1, j0 = jb * 128;
+            if (kPass == 2) {
+                const int j = j0 + wt;
+                const float z = (j < S) ? sc_z[size_t(rowbase) + j] : 1.f;
+                ctl->invz[s][wt] = (z > 0.f) ? 1.f / z : 0.f;
+                named_bar_sync(1, 128);
+            }
+            ok = gram_wait(ctl, &ctl->tfull[s], uint32_t(jb >> 1) & 1u, status);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after();
+            const bool interior = (j0 + 128 <= S) && (j0 != i0);
+#pragma unroll
+            for (int ch = 0; ch < 4; ++ch) {
+                float v[32];
+                tmem_ld32(lane_addr + s * 128 + ch * 32, v);
+                if (interior) {
+                    float e0 = 0.f, e1 = 0.f;
+#pragma unroll
+                    for (int jj = 0; jj < 32; jj += 2) {
+                        if (kPass == 1) {
+                            e0 += ex2f(v[jj] * kLog2e);
+                            e1 += ex2f(v[jj + 1] * kLog2e);
+                        } else {
+                            e0 = fmaf(ex2f(v[jj] * kLog2e), ctl->invz[s][ch * 32 + jj], e0);
+                            e1 = fmaf(ex2f(v[jj + 1] * kLog2e), ctl->invz[s][ch * 32 + jj + 1], e1);
+                        }
+                    }
+                    accum += e0 + e1;
+                    if (kPass == 1 && j0 > i0) {
+#pragma unroll
+                        for (int jj = 0; jj < 32; ++jj) mx = fmaxf(mx, v[jj]);
+                    }
+                } else {
+#pragma unroll
+                    for (int jj = 0; jj < 32; ++jj) {
+                        const int j = j0 + ch * 32 + jj;
+                        if (j < S && j != i) {
+                            const float e = ex2f(v[jj] * kLog2e);
+                            if (kPass == 1) {
+                                accum += e;
+                                if (j > i) mx = fmaxf(mx, v[jj]);
+                            } else {
+                                accum = fmaf(e, ctl->invz[s][ch * 32 + jj], accum);
+                            }
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&ctl->tempty[s]);
+        }
+        if (ok && i < S) {
+            const size_t o = size_t(rowbase) + i;
             if (kPass == 1) {
-                accum += e;
-                if (j > i) mx = fmaxf(mx, g);
+                sc_z[o] = accum;
+                sent_lam[o] = (mx > tau) ? mx : 0.f;
             } else {
-                accum += e / sc_z[size_t(slab) * max_sent + j];
+                const float red = accum / float(S);
+                sent_red[o] = red;
+                sent_score[o] = sigma * sent_imp[o] - (1.f - sigma) * red - sent_lam[o];
             }
         }
     }
-#pragma unroll
-    for (int d = 16; d; d >>= 1) {
-        accum += __shfl_xor_sync(0xffffffffu, accum, d);
-        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, d));
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, 256);
     }
-    if (tj == 0 && i < S) {
-        const size_t o = size_t(slab) * max_sent + i;
-        if (kPass == 1) {
-            sc_z[o] = accum;
-            sent_lam[o] = (mx > tau) ? mx : 0.f;
-        } else {
-            const float red = accum / float(S);
-            sent_red[o] = red;
-            sent_score[o] = sigma * sent_imp[o] - (1.f - sigma) * red - sent_lam[o];
-        }
-    }
+}
+
+template <int kSweep, int kN>
+static int launch_sweep(const CUtensorMap& mapK, const CUtensorMap& mapQ, const SweepArgs& a, int grid, size_t smem,
+                        cudaStream_t st) {
+    auto kern = score_sweep_kernel<kSweep, kN>;
+    SKIPKV_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
+    kern<<<grid, kSweep == 1 ? kSw1Threads : kSw2Threads, smem, st>>>(mapK, mapQ, a);
+    SKIPKV_CUDA(cudaGetLastError());
+    return SKIPKV_OK;
 }
 
 }  // namespace skipkv
@@ -307,45 +703,71 @@ extern "C" int skipkv_score(const skipkv_shape* shape, const skipkv_params* para
     if (shape->max_sent <= 0) return SKIPKV_OK;
     const WsLayout L = make_layout(*shape);
     uint8_t* w = static_cast<uint8_t*>(ws);
-    float2* sc_part = reinterpret_cast<float2*>(w + L.sc_part);
-    float* sc_lse = reinterpret_cast<float*>(w + L.sc_lse);
+    uint32_t* status = &reinterpret_cast<Header*>(w + L.header)->status;
     float* sc_tok = reinterpret_cast<float*>(w + L.sc_tokimp);
-    float* sc_vbar = reinterpret_cast<float*>(w + L.sc_vbar);
+    float* vsum = reinterpret_cast<float*>(w + L.sc_vsum);
+    __nv_bfloat16* vbar_hi = reinterpret_cast<__nv_bfloat16*>(w + L.sc_vbar_hi);
+    __nv_bfloat16* vbar_lo = reinterpret_cast<__nv_bfloat16*>(w + L.sc_vbar_lo);
     float* sc_z = reinterpret_cast<float*>(w + L.sc_z);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const int Hq = shape->n_q_heads, Hk = shape->n_kv_heads;
-    const uint8_t* Kb = static_cast<const uint8_t*>(K);
-    const uint8_t* Qb = static_cast<const uint8_t*>(q_win);
+    const int Hq = shape->n_q_heads, Hk = shape->n_kv_heads, n = L.group;
 
+    CUtensorMap mapK, mapQ, mapHi, mapLo;
+    if (int rc = tmap_rows(&mapK, K, uint64_t(shape->total_rows), 128)) return rc;
+    if (int rc = tmap_qwin(&mapQ, q_win, uint64_t(shape->batch) * Hq, uint32_t(shape->window), uint32_t(L.sc_wb), uint32_t(n)))
+        return rc;
+    const uint64_t vrows = uint64_t(L.slabs) * uint64_t(shape->max_sent);
+    if (int rc = tmap_rows(&mapHi, vbar_hi, vrows, 128)) return rc;
+    if (int rc = tmap_rows(&mapLo, vbar_lo, vrows, 128)) return rc;
+
+    SweepArgs a{};
+    a.Hq = Hq; a.Hk = Hk; a.window = shape->window; a.n_slabs = L.slabs; a.max_cap = shape->max_cap;
+    a.max_sent = shape->max_sent; a.RB = L.sc_rb; a.WB = L.sc_wb;
+    a.slab_off = shape->slab_off; a.cap = shape->cap; a.kv_len = kv_len; a.sent_off = sent_off; a.n_sent = n_sent;
+    a.sc_part = reinterpret_cast<float2*>(w + L.sc_part);
+    a.tok_imp_user = tok_imp; a.tok_imp_ws = sc_tok; a.vsum = vsum; a.status = status;
+    const size_t fixed = 1024 + size_t(a.RB) * kOpBytes + sizeof(SweepCtl) + size_t(L.slabs + 1) * 4;
+    const size_t max_smem = 227 * 1024;
+    if (fixed + kOpBytes > max_smem) return SKIPKV_ERR_UNSUPPORTED;
+    int stages = int((max_smem - fixed) / kOpBytes);
+    if (stages > kSwMaxStages) stages = kSwMaxStages;
+    a.stages = stages;
+    const size_t smem = fixed + size_t(stages) * kOpBytes;
+    int grid = num_sms();
+    if (grid > L.dec_max_ctas) grid = L.dec_max_ctas;
+
+    SKIPKV_CUDA(cudaMemsetAsync(vsum, 0, size_t(L.slabs) * shape->max_sent * kHeadDim * 4, st));
+    if (int rc = launch_sweep<1, 1>(mapK, mapQ, a, grid, smem, st)) return rc;
+    int rc = SKIPKV_ERR_UNSUPPORTED;
+    switch (n) {
+        case 1: rc = launch_sweep<2, 1>(mapK, mapQ, a, grid, smem, st); break;
+        case 2: rc = launch_sweep<2, 2>(mapK, mapQ, a, grid, smem, st); break;
+        case 3: rc = launch_sweep<2, 3>(mapK, mapQ, a, grid, smem, st); break;
+        case 4: rc = launch_sweep<2, 4>(mapK, mapQ, a, grid, smem, st); break;
+        case 5: rc = launch_sweep<2, 5>(mapK, mapQ, a, grid, smem, st); break;
+        case 6: rc = launch_sweep<2, 6>(mapK, mapQ, a, grid, smem, st); break;
+        case 7: rc = launch_sweep<2, 7>(mapK, mapQ, a, grid, smem, st); break;
+        case 8: rc = launch_sweep<2, 8>(mapK, mapQ, a, grid, smem, st); break;
+        default: break;
+    }
+    if (rc) return rc;
     {
-        const int threads = L.qrows >= 256 ? 256 : ((L.qrows + 31) / 32) * 32;
-        dim3 grid(L.sc_chunks, L.slabs, (L.qrows + 255) / 256);
-        score_sweep1_kernel<<<grid, threads, 0, st>>>(Hq, Hk, shape->window, L.qrows, L.sc_chunks, shape->slab_off,
-                                                      shape->cap, Kb, Qb, kv_len, sc_part);
+        dim3 pgrid((shape->max_sent + 7) / 8, L.slabs);
+        score_pool_kernel<<<pgrid, 256, 0, st>>>(Hk, shape->max_sent, shape->max_cap, shape->cap, kv_len, sent_off,
+                                                 n_sent, params->eps, sc_tok, vsum, sent_imp, vbar_hi, vbar_lo);
         SKIPKV_CUDA(cudaGetLastError());
     }
-    score_lse_kernel<<<L.slabs, 128, 0, st>>>(L.qrows, L.sc_chunks, kv_len, sc_part, sc_lse);
-    SKIPKV_CUDA(cudaGetLastError());
     {
-        dim3 grid((shape->max_cap + kS2Tokens - 1) / kS2Tokens, L.slabs);
-        score_sweep2_kernel<<<grid, kS2Tokens, 0, st>>>(Hq, Hk, shape->window, L.qrows, shape->max_cap,
-                                                        shape->slab_off, shape->cap, Kb, Qb, kv_len, sc_lse, tok_imp,
-                                                        sc_tok);
+        dim3 ggrid((shape->max_sent + 127) / 128, L.slabs);
+        SKIPKV_CUDA(cudaFuncSetAttribute(score_gram_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kGramSmem)));
+        SKIPKV_CUDA(cudaFuncSetAttribute(score_gram_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kGramSmem)));
+        score_gram_kernel<1><<<ggrid, kGramThreads, kGramSmem, st>>>(mapHi, mapLo, shape->max_sent, n_sent, params->sigma,
+                                                                    params->tau, sc_z, sent_imp, sent_red, sent_lam,
+                                                                    sent_score, status);
         SKIPKV_CUDA(cudaGetLastError());
-    }
-    {
-        dim3 grid((shape->max_sent + 7) / 8, L.slabs);
-        score_pool_kernel<<<grid, 256, 0, st>>>(Hk, shape->max_sent, shape->max_cap, shape->slab_off, shape->cap, Kb,
-                                                kv_len, sent_off, n_sent, params->eps, sc_tok, sent_imp, sc_vbar);
-        SKIPKV_CUDA(cudaGetLastError());
-    }
-    {
-        dim3 grid((shape->max_sent + 31) / 32, L.slabs);
-        score_gram_kernel<1><<<grid, 1024, 0, st>>>(shape->max_sent, n_sent, params->sigma, params->tau, sc_vbar, sc_z,
-                                                    sent_imp, sent_red, sent_lam, sent_score);
-        SKIPKV_CUDA(cudaGetLastError());
-        score_gram_kernel<2><<<grid, 1024, 0, st>>>(shape->max_sent, n_sent, params->sigma, params->tau, sc_vbar, sc_z,
-                                                    sent_imp, sent_red, sent_lam, sent_score);
+        score_gram_kernel<2><<<ggrid, kGramThreads, kGramSmem, st>>>(mapHi, mapLo, shape->max_sent, n_sent, params->sigma,
+                                                                    params->tau, sc_z, sent_imp, sent_red, sent_lam,
+                                                                    sent_score, status);
         SKIPKV_CUDA(cudaGetLastError());
     }
     return SKIPKV_OK;
