@@ -33,7 +33,7 @@ struct WsLayout {
     size_t cp_run_dst;     // int32  [slabs][max_sent+1]  first destination token; [nruns] = new_len
     size_t dec_cnt;        // uint32 [slabs]              partials that arrived (self-resetting)
     size_t dec_part;       // float  [max_ctas + slabs][group][130]
-    size_t sc_part;        // float2 [(max_ctas + slabs) * 2][sc_rb * 128]  (max, sum) of a CTA's part of a slab
+    size_t sc_part;        // float2 [(max_ctas + slabs) * 4][sc_rb * 128]  (max, sum) of a CTA's part of a slab
     size_t sc_tokimp;      // float  [slabs][max_cap]
     size_t sc_vsum;        // float  [slabs][max_sent][128]  per-sentence sums of key rows
     size_t sc_vbar_hi;     // bf16   [slabs][max_sent][128]  normalised mean key, high part
@@ -69,7 +69,7 @@ inline WsLayout make_layout(const skipkv_shape& s) {
     L.cp_run_dst = take(slabs * (ms + 1) * 4);
     L.dec_cnt = take(slabs * 4);
     L.dec_part = take((size_t(L.dec_max_ctas) + slabs) * L.group * 130 * 4);
-    L.sc_part = take((size_t(L.dec_max_ctas) + slabs) * 2 * size_t(L.sc_rb) * 128 * 8);
+    L.sc_part = take((size_t(L.dec_max_ctas) + slabs) * 4 * size_t(L.sc_rb) * 128 * 8);
     L.sc_tokimp = take(slabs * size_t(s.max_cap > 0 ? s.max_cap : 1) * 4);
     L.sc_vsum = take(slabs * ms * kHeadDim * 4);
     L.sc_vbar_hi = take(slabs * ms * kHeadDim * 2);

@@ -15,8 +15,8 @@
 //
 // Both sweeps are persistent, warp-specialised kernels, one CTA per SM: a TMA warp streams
 // 128-token key tiles (and the group's query block) into shared memory, one thread issues
-// tcgen05.mma into a ring of four tensor-memory accumulators, two warpgroups of epilogue warps
-// alternate over the tiles, and (sweep 2) one more warpgroup pools the key rows.  Work is the list of
+// tcgen05.mma into a ring of four tensor-memory accumulators, several warpgroups of epilogue warps
+// take the tiles round-robin, and (sweep 2) one more warpgroup pools the key rows.  Work is the list of
 // 128-token tiles over all slabs cut into equal contiguous ranges, so ragged slabs balance.
 //
 // Query rows of a group are staged as blocks of WB = floor(128/n) window positions x n heads
@@ -32,8 +32,10 @@ namespace skipkv {
 constexpr int kAccBufs = 4;             // tensor-memory accumulators of 128 columns
 constexpr int kMaxRB = 4;               // query blocks per group
 constexpr int kSwMaxStages = 6;
-constexpr int kSw1Threads = 10 * 32;    // TMA, MMA, 8 epilogue warps
-constexpr int kSw2Threads = 14 * 32;    // + 4 pooling warps
+constexpr int kSw1Groups = 4;           // epilogue warpgroups of sweep 1
+constexpr int kSw2Groups = 3;           // epilogue warpgroups of sweep 2 (plus one pooling warpgroup)
+constexpr int kSw1Threads = (2 + 4 * kSw1Groups) * 32;        // TMA warp, MMA warp, epilogue warps
+constexpr int kSw2Threads = (2 + 4 * kSw2Groups + 4) * 32;    // + 4 pooling warps
 constexpr float kLog2e = 1.4426950408889634f;
 
 __device__ __forceinline__ float ex2f(float x) {
@@ -49,7 +51,7 @@ struct SweepCtl {                       // barriers and small shared state, afte
     uint32_t tmem_base;
     int abort_flag;
     uint32_t wsum[16];
-    alignas(16) float neg_lse[2][kMaxRB * 128];   // sweep 2: one copy per epilogue warpgroup (read as float4)
+    alignas(16) float neg_lse[kSw2Groups][kMaxRB * 128];   // sweep 2: one copy per epilogue warpgroup (read as float4)
 };
 static_assert(offsetof(SweepCtl, neg_lse) % 16 == 0, "neg_lse is read with 16-byte loads");
 
@@ -60,7 +62,7 @@ struct SweepArgs {
     const int32_t* kv_len;
     const int32_t* sent_off;
     const int32_t* n_sent;
-    float2* sc_part;                    // [(cta + slab) * 2 + warpgroup][RB * 128] (max, sum)
+    float2* sc_part;                    // [(cta + slab) * kSw1Groups + warpgroup][RB * 128] (max, sum)
     float* tok_imp_user;
     float* tok_imp_ws;
     float* vsum;                        // [slabs][max_sent][128] sums of key rows
@@ -149,6 +151,7 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_consta
                    const SweepArgs a) {
     extern __shared__ uint8_t sweep_smem_raw[];
     constexpr int kThreads = kSweep == 1 ? kSw1Threads : kSw2Threads;
+    constexpr int kGroups = kSweep == 1 ? kSw1Groups : kSw2Groups;
     const uint32_t raw = smem_u32(sweep_smem_raw);
     uint8_t* tiles = sweep_smem_raw + (((raw + 1023u) & ~1023u) - raw);          // 1024-byte aligned
     uint8_t* qbuf = tiles + size_t(a.stages) * kOpBytes;
@@ -286,9 +289,9 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_consta
                 if (++stage == a.stages) { stage = 0; ++lap; }
             }
         }
-    } else if (warp < 10) {
+    } else if (warp < 2 + 4 * kGroups) {
         // ------------------------------------------------------------------ epilogue warpgroups
-        const int g = (warp - 2) >> 2;                       // warpgroup: tiles t_begin + g, + g + 2, ...
+        const int g = (warp - 2) >> 2;                       // warpgroup: tiles t_begin + g, + g + kGroups, ...
         const int quarter = warp & 3;                        // tensor-memory lanes this warp may read
         const int row = quarter * 32 + lane;
         const uint32_t lane_addr = tmem_base + (uint32_t(quarter * 32) << 16);
@@ -302,7 +305,7 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_consta
                 float m[kMaxRB], l[kMaxRB];
 #pragma unroll
                 for (int k = 0; k < kMaxRB; ++k) { m[k] = -INFINITY; l[k] = 0.f; }
-                for (; t_begin + tl < seg_end; tl += 2) {
+                for (; t_begin + tl < seg_end; tl += kGroups) {
                     const int t = t_begin + tl;
                     const int valid = min(128, N - (t - pref[slab]) * 128);
 #pragma unroll
@@ -322,7 +325,7 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_consta
                         }
                     }
                 }
-                float2* rec = a.sc_part + (size_t(cta + slab) * 2 + g) * (size_t(RB) * 128);
+                float2* rec = a.sc_part + (size_t(cta + slab) * kSw1Groups + g) * (size_t(RB) * 128);
 #pragma unroll
                 for (int k = 0; k < kMaxRB; ++k)
                     if (k < RB) rec[k * 128 + row] = make_float2(m[k], l[k]);
@@ -334,7 +337,7 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_consta
             int N = 0;
             size_t row0 = 0;
             bool have = false;
-            for (; tl < ntl; tl += 2) {
+            for (; tl < ntl; tl += kGroups) {
                 const int t = t_begin + tl;
                 if (!have || pref[slab + 1] <= t) {
                     while (pref[slab + 1] <= t) ++slab;
@@ -343,8 +346,8 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_consta
                     row0 = slab_row0(a.slab_off, a.cap, Hk, slab / Hk, slab % Hk);
                     // log-sum-exp of every query row of this slab from the sweep-1 records
                     const int fc = pref[slab] / per_cta, lc = (pref[slab + 1] - 1) / per_cta;
-                    const float2* r0 = a.sc_part + size_t(fc + slab) * 2 * (size_t(RB) * 128);
-                    const int n_part = (lc - fc + 1) * 2;
+                    const float2* r0 = a.sc_part + size_t(fc + slab) * kSw1Groups * (size_t(RB) * 128);
+                    const int n_part = (lc - fc + 1) * kSw1Groups;
                     named_bar_sync(2 + g, 128);              // previous readers of nl are done
                     for (int k = 0; k < RB; ++k) {
                         float M = -INFINITY;
@@ -385,8 +388,13 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_consta
         }
     } else if (kSweep == 2) {
         // ------------------------------------------------------------------ pooling warps: per-sentence sums of key rows
-        const int pt = tid - 320, g2 = pt >> 6, c2 = pt & 63;          // two groups of 64 rows; 2 channels per thread
-        const int half = c2 >> 5, chunk = (c2 & 31) >> 2, within = c2 & 3;
+        // warp pw owns rows [32 pw, 32 pw + 32) of every tile; a lane owns 4 channels (8 bytes) of a row
+        const int pw = warp - (2 + 4 * kGroups);
+        const int half = lane >> 4, chunk = (lane & 15) >> 1, sub = (lane & 1) * 8;
+        const int ch0 = half * 64 + (lane & 15) * 4;                   // first channel of this lane
+        int swz[8];                                                    // byte offset of this lane's chunk in row i of 8
+#pragma unroll
+        for (int i = 0; i < 8; ++i) swz[i] = i * 128 + ((chunk ^ i) << 4);
         int slab = slab0, S = 0, N = 0, cur = -1;
         const int32_t* so = a.sent_off;
         bool ok = true, have = false;
@@ -404,7 +412,7 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_consta
                 cur = -1;
             }
             const int tok0 = (t - pref[slab]) * 128;
-            const int r_lo = g2 * 64, r_hi = min(r_lo + 64, N - tok0);
+            const int r_lo = pw * 32, r_hi = min(r_lo + 32, N - tok0);
             if (S > 0 && r_lo < r_hi) {
                 const int tk = tok0 + r_lo;
                 if (cur < 0) {
@@ -417,21 +425,39 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_consta
                 } else {
                     while (cur + 1 < S && so[cur + 1] <= tk) ++cur;
                 }
-                const uint8_t* colbase = tiles + size_t(stage) * kOpBytes + half * kOpHalfBytes + within * 4;
+                const uint8_t* colbase = tiles + size_t(stage) * kOpBytes + half * kOpHalfBytes + sub;
+                auto ld = [&](int r) {
+                    return *reinterpret_cast<const uint2*>(colbase + r * 128 + ((chunk ^ (r & 7)) << 4));
+                };
                 int r = r_lo;
                 while (r < r_hi) {
                     int e = r_hi;
                     if (cur + 1 < S) e = min(e, so[cur + 1] - tok0);
                     if (e > r) {
-                        float a0 = 0.f, a1 = 0.f;
-                        for (; r < e; ++r) {
-                            const uint32_t u =
-                                *reinterpret_cast<const uint32_t*>(colbase + r * 128 + ((chunk ^ (r & 7)) << 4));
-                            a0 += bf16lo(u);
-                            a1 += bf16hi(u);
+                        float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+                        for (; (r & 7) && r < e; ++r) {          // up to a swizzle-period boundary
+                            const uint2 u = ld(r);
+                            a0 += bf16lo(u.x); a1 += bf16hi(u.x);
+                            a2 += bf16lo(u.y); a3 += bf16hi(u.y);
                         }
-                        atomicAdd(reinterpret_cast<float2*>(a.vsum + (size_t(slab) * a.max_sent + cur) * kHeadDim) + c2,
-                                  make_float2(a0, a1));
+                        for (; r + 8 <= e; r += 8) {             // r % 8 == 0: the offsets are the precomputed ones
+                            const uint8_t* rp = colbase + r * 128;
+                            uint2 u[8];
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) u[i] = *reinterpret_cast<const uint2*>(rp + swz[i]);
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) {
+                                a0 += bf16lo(u[i].x); a1 += bf16hi(u[i].x);
+                                a2 += bf16lo(u[i].y); a3 += bf16hi(u[i].y);
+                            }
+                        }
+                        for (; r < e; ++r) {
+                            const uint2 u = ld(r);
+                            a0 += bf16lo(u.x); a1 += bf16hi(u.x);
+                            a2 += bf16lo(u.y); a3 += bf16hi(u.y);
+                        }
+                        atomicAdd(reinterpret_cast<float4*>(a.vsum + (size_t(slab) * a.max_sent + cur) * kHeadDim + ch0),
+                                  make_float4(a0, a1, a2, a3));
                     }
                     if (r < r_hi) ++cur;                     // the piece ended on a sentence boundary
                 }
