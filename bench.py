@@ -8,7 +8,9 @@ attention (with the fused steering add) over one layer of the Llama-8B-shaped wo
 
 Prints ONE JSON line.  `value` is the eviction time (score+select+compact) per layer in
 microseconds with inputs resident in HBM; the decode-attention bandwidth and the per-step
-rooflines ride along in the same line.  With N > 1 every rank runs an independent replica of
+rooflines ride along in the same line.  A step runs every leg over `--layers` independently
+seeded layers back to back (the order of a multi-layer eviction pass and of a decode step), so
+no launch finds its K/V in L2 and a leg's time divided by the layer count is the average launch.  With N > 1 every rank runs an independent replica of
 the workload (the path has no exchange step); the time is the max over ranks and the value is
 that time divided by the N layers processed.
 """
@@ -33,7 +35,7 @@ from paper_2512_07993_b200 import workloads as W  # noqa: E402
 
 METRIC = "SkipKV compress+compact µs/layer and decode-attn HBM GB/s, 32K ctx, batch 10"
 UNIT = "us/layer (score+select+compact); decode-attn GB/s in decode_attn_gbs"
-LAUNCHES_PER_STEP = {"score": 6, "select": 1, "compact": 2, "decode_attn": 1}
+LAUNCHES_PER_STEP = {"score": 5, "select": 1, "compact": 2, "decode_attn": 1}      # kernels per layer
 
 
 def measured_peaks():
@@ -60,6 +62,7 @@ class ClockSampler:
         self.index, self.lines, self.proc = index, [], None
 
     def start(self):
+        self.t_start = time.time()
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
                                           "-i", str(self.index), "-lms", "100"], stdout=subprocess.PIPE, text=True)
@@ -74,8 +77,9 @@ class ClockSampler:
     def stop(self, t0, t1):
         if self.proc is None:
             return None
-        time.sleep(0.15)
-        self.proc.terminate()
+        if self.proc.poll() is None:
+            time.sleep(0.15)
+            self.proc.terminate()
         sm, mx, reasons = [], [], set()
         for ts, line in self.lines:
             f = [x.strip() for x in line.split(",")]
@@ -90,7 +94,8 @@ class ClockSampler:
                     reasons.add(name)
         if not sm:
             return None
-        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons), "samples": len(sm)}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons), "samples": len(sm),
+                "window": "warm-up + timed region" if t0 < self.t_start + 1e-3 else "timed region"}
 
 
 def oracle_shape(L):
@@ -164,11 +169,12 @@ def run_reference(args, rank):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=30)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="skipkv", choices=["skipkv", "reference"])
     ap.add_argument("--config", type=int, default=2, help="workload index (2 = the headline configuration)")
     ap.add_argument("--batch", type=int, default=0, help="override the number of sequences (profiling captures)")
+    ap.add_argument("--layers", type=int, default=4, help="layers (independent K/V buffers) each leg of a step runs over")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -194,34 +200,46 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
 
     cfg = W.config(args.config, batch=args.batch) if args.batch else W.config(args.config)
-    L = W.make_layer(cfg)
-    D = B.DeviceLayer(L)
-    pristine = {k: getattr(D, k).clone() for k in ("K", "V", "sent_off", "sent_id", "n_sent", "kv_len", "hidden")}
+    NL = max(1, args.layers)
+    # NL independently seeded layers of the workload, each with its own K/V: every leg of a step runs
+    # over all of them back to back, so a launch never finds its inputs in L2 (1 GB per layer)
+    Ls = [W.make_layer(cfg, layer=l) for l in range(NL)]
+    Ds = [B.DeviceLayer(L) for L in Ls]
+    L, D = Ls[0], Ds[0]
+    keys = ("K", "V", "sent_off", "sent_id", "n_sent", "kv_len", "hidden")
+    pristine = [{k: getattr(Dl, k).clone() for k in keys} for Dl in Ds]
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    clean = torch.ones(256 << 20, dtype=torch.uint8, device="cuda")
 
     def restore():
-        for k, v in pristine.items():
-            getattr(D, k).copy_(v)
-        flush.fill_(1)                      # evict whatever the restore left in L2
+        for Dl, pr in zip(Ds, pristine):
+            for k, v in pr.items():
+                getattr(Dl, k).copy_(v)
+        flush.fill_(1)                      # evict whatever the restore left in L2 ...
+        clean.sum()                         # ... then read a clean buffer: no dirty lines are left to write back
 
     legs = ("score", "select", "compact", "decode_attn")
     ev = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(args.steps)]
 
     def step(events=None):
         rec = (lambda i: events[i].record()) if events else (lambda i: None)
-        rec(0); D.score()
-        rec(1); D.select()
-        rec(2); D.compact()
-        rec(3); D.decode_attn(steer=True)
+        rec(0)
+        for Dl in Ds: Dl.score()
+        rec(1)
+        for Dl in Ds: Dl.select()
+        rec(2)
+        for Dl in Ds: Dl.compact()
+        rec(3)
+        for Dl in Ds: Dl.decode_attn(steer=True)
         rec(4)
 
+    clocks = ClockSampler(local_rank); clocks.start()      # nvidia-smi needs a moment to deliver its first sample
     for _ in range(args.warmup):
         restore(); step()
     torch.cuda.synchronize()
-    D.status()
+    for Dl in Ds: Dl.status()
     if dist: dist.barrier()
     torch.cuda.synchronize()
-    clocks = ClockSampler(local_rank); clocks.start()
     t0 = time.time()
     for i in range(args.steps):
         restore(); step(ev[i])
@@ -230,13 +248,16 @@ def main():
     torch.cuda.synchronize()
     t1 = time.time()
     clk = clocks.stop(t0, t1)
-    D.status()
+    if clk is None:                 # timed region shorter than the sampling period: use the warm-up samples too (same load)
+        clk = clocks.stop(clocks.t_start, t1)
+    for Dl in Ds: Dl.status()
 
-    per = {leg: [ev[i][k].elapsed_time(ev[i][k + 1]) * 1e3 for i in range(args.steps)] for k, leg in enumerate(legs)}
+    # per-launch (= per-layer) times: a leg's elapsed time over its NL back-to-back calls
+    per = {leg: [ev[i][k].elapsed_time(ev[i][k + 1]) * 1e3 / NL for i in range(args.steps)] for k, leg in enumerate(legs)}
     us = {leg: statistics.mean(v) for leg, v in per.items()}
     us_med = {leg: statistics.median(v) for leg, v in per.items()}
     evict_us = us["score"] + us["select"] + us["compact"]
-    step_ms = sum(us.values()) / 1e3
+    step_ms = sum(us.values()) * NL / 1e3
     if dist:
         tt = torch.tensor([evict_us, step_ms, us["decode_attn"]], device="cuda", dtype=torch.float64)
         dist.all_reduce(tt, op=dist.ReduceOp.MAX)
@@ -244,13 +265,13 @@ def main():
     else:
         dec_us_max = us["decode_attn"]
 
-    # algorithmic bytes from the actual lengths
-    kv0 = L["kv_len"].astype(np.int64)
-    kv1 = D.kv_len.cpu().numpy().astype(np.int64)
+    # algorithmic bytes per layer from the actual lengths (mean over the NL layers)
+    kv0 = np.stack([Ll["kv_len"].astype(np.int64) for Ll in Ls])
+    kv1 = np.stack([Dl.kv_len.cpu().numpy().astype(np.int64) for Dl in Ds])
     row = 2 * cfg.head_dim
-    bytes_alg = {"score": int(kv0.sum()) * row,                      # K read once
-                 "compact": int(kv1.sum()) * row * 2 * 2,            # kept K and V rows read and written
-                 "decode_attn": int(kv1.sum()) * row * 2}            # live K and V rows read once
+    bytes_alg = {"score": int(kv0.sum()) * row // NL,                 # K read once
+                 "compact": int(kv1.sum()) * row * 2 * 2 // NL,       # kept K and V rows read and written
+                 "decode_attn": int(kv1.sum()) * row * 2 // NL}       # live K and V rows read once
     peaks = measured_peaks()
     traffic = ncu_traffic()
     roof = {}
@@ -267,17 +288,20 @@ def main():
             "vs_baseline": None, "dtype": "bf16 storage, f32 arithmetic", "data": "synthetic",
             "config": {"workload": f"configs[{args.config - 1}]: {cfg.name}", "batch": cfg.batch,
                        "kv_heads": cfg.n_kv_heads, "q_heads": cfg.n_q_heads, "head_dim": cfg.head_dim,
-                       "window": cfg.window, "budget": cfg.budget, "tokens_before": int(kv0.sum() // cfg.n_kv_heads),
-                       "tokens_after": int(kv1.sum() // cfg.n_kv_heads), "layers_per_step": 1,
-                       "l2": "256 MiB flush buffer written between iterations; inputs (1 GB) exceed L2",
+                       "window": cfg.window, "budget": cfg.budget,
+                       "tokens_before": int(kv0.sum() // cfg.n_kv_heads // NL),
+                       "tokens_after": int(kv1.sum() // cfg.n_kv_heads // NL), "layers_per_step": NL,
+                       "order": "each leg (score, select, compact, decode) runs over all layers back to back; "
+                                "per-layer time = leg time / layers",
+                       "l2": "256 MiB written then 256 MiB read between iterations; each layer's inputs (1 GB) exceed L2",
                        "replicas": world},
             "us": us, "decode_attn_us": dec_us_max, "decode_attn_gbs": bytes_alg["decode_attn"] / (dec_us_max * 1e-6) / 1e9,
             "roofline": dict(roof[dominant], kernel=dominant), "roofline_by_step": roof,
-            "gpu_launches": sum(LAUNCHES_PER_STEP.values()) * args.steps, "clocks": clk}
+            "gpu_launches": sum(LAUNCHES_PER_STEP.values()) * NL * args.steps, "clocks": clk}
 
     # ---- end to end through the C ABI with host buffers (pinned), copies inside the timed region
     if not args.no_e2e:
-        host_in = {k: pristine[k].cpu().pin_memory() for k in ("K", "V", "sent_off", "sent_id", "n_sent", "kv_len", "hidden")}
+        host_in = {k: pristine[0][k].cpu().pin_memory() for k in keys}
         host_in["q_win"] = D.q_win.cpu().pin_memory(); host_in["q"] = D.q.cpu().pin_memory()
         outs = ("out", "kv_len", "n_sent", "sent_off", "sent_id", "hidden")
         host_out = {k: torch.empty_like(getattr(D, k), device="cpu").pin_memory() for k in outs}
