@@ -27,7 +27,7 @@ namespace skipkv {
 constexpr int kSegRows = 256;                       // rows per segment (64 KB of shared memory)
 constexpr int kSegBytes = kSegRows * kRowBytes;
 constexpr int kMoveThreads = 128;
-constexpr int kPlanThreads = 256;
+constexpr int kPlanThreads = 1024;
 
 // exclusive block scan of three ints at once; returns the block totals through tot[]
 __device__ __forceinline__ void block_scan3(int v0, int v1, int v2, int& e0, int& e1, int& e2, int tot[3],
