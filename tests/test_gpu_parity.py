@@ -49,6 +49,13 @@ def cases():
         "ragged": W.config(1, name="ragged", batch=3, ctx_lo=700, ctx_hi=2100, budget=1500, seed=77, dup_rate=0.3),
         "group5": W.config(0, name="group5", n_q_heads=10, n_kv_heads=2, window=12, ctx_lo=500, ctx_hi=900,
                            budget=333, seed=5),
+        # the stress configuration's group shape: 5 heads per KV head, 64-query window (three query blocks per group)
+        "group5-window64": W.config(0, name="group5-window64", n_q_heads=10, n_kv_heads=2, window=64, ctx_lo=900,
+                                    ctx_hi=1700, budget=600, seed=9, sent_dist="geometric", geo_mean_extra=20.0,
+                                    sent_hi=128, dup_rate=0.4),
+        # eight heads per KV head with a 64-query window: four query blocks, the most the kernels take
+        "group8-window64": W.config(0, name="group8-window64", batch=1, n_q_heads=16, n_kv_heads=2, window=64,
+                                    ctx_lo=700, ctx_hi=700, budget=300, seed=10),
     }
 
 
