@@ -47,7 +47,10 @@ __device__ __forceinline__ float ex2f(float x) {
 struct SweepCtl {                       // barriers and small shared state, after the tile buffers
     uint64_t full[kSwMaxStages], empty[kSwMaxStages];
     uint64_t qfull, qempty;
-    uint64_t tfull[kAccBufs], tempty[kAccBufs];
+    // "accumulator ready" barriers are per epilogue warpgroup (a ring of 4 per group, indexed by the group's own item
+    // count), so every barrier has one consumer that sees its phases in order; a barrier per accumulator would be
+    // waited on by different groups in turn, and a group polling for a later phase could pass on an earlier one.
+    uint64_t tfull[4][4], tempty[kAccBufs];
     uint32_t tmem_base;
     int abort_flag;
     uint32_t wsum[16];
@@ -170,7 +173,9 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_consta
         }
         mbar_init(&ctl->qfull, 1);
         mbar_init(&ctl->qempty, 1);
-        for (int b = 0; b < kAccBufs; ++b) { mbar_init(&ctl->tfull[b], 1); mbar_init(&ctl->tempty[b], 4); }
+        for (int b = 0; b < kAccBufs; ++b) mbar_init(&ctl->tempty[b], 4);
+        for (int g = 0; g < 4; ++g)
+            for (int j = 0; j < 4; ++j) mbar_init(&ctl->tfull[g][j], 1);
         ctl->abort_flag = 0;
         mbar_fence_init();
         tmap_prefetch(&mapK);
@@ -282,7 +287,10 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_consta
                     const uint32_t q_smem = smem_u32(qbuf + size_t(k) * kOpBytes);
                     if (kSweep == 1) umma_tile_128x128x128(tmem_base + buf * 128, q_smem, k_smem, false);
                     else             umma_tile_128x128x128(tmem_base + buf * 128, k_smem, q_smem, false);
-                    umma_commit(&ctl->tfull[buf]);
+                    {
+                        const int ti = t - t_begin, gj = (ti / kGroups) * RB + k;     // the owning group's item count
+                        umma_commit(&ctl->tfull[ti % kGroups][gj & 3]);
+                    }
                 }
                 umma_commit(&ctl->empty[stage]);
                 if (t + 1 == t_end || pref[slab + 1] <= t + 1) umma_commit(&ctl->qempty);
@@ -312,7 +320,8 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_consta
                     for (int k = 0; k < kMaxRB; ++k) {
                         if (k < RB && ok) {
                             const int it = tl * RB + k, buf = it & (kAccBufs - 1);
-                            ok = ctl_wait(ctl, &ctl->tfull[buf], uint32_t(it / kAccBufs) & 1u, a.status);
+                            const int gj = (tl / kGroups) * RB + k;
+                            ok = ctl_wait(ctl, &ctl->tfull[g][gj & 3], uint32_t(gj >> 2) & 1u, a.status);
                             ok = __all_sync(0xffffffffu, ok);
                             if (ok) {
                                 tc_fence_after();
@@ -366,7 +375,8 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_consta
                 for (int k = 0; k < kMaxRB; ++k) {
                     if (k < RB && ok) {
                         const int it = tl * RB + k, buf = it & (kAccBufs - 1);
-                        ok = ctl_wait(ctl, &ctl->tfull[buf], uint32_t(it / kAccBufs) & 1u, a.status);
+                        const int gj = (tl / kGroups) * RB + k;
+                        ok = ctl_wait(ctl, &ctl->tfull[g][gj & 3], uint32_t(gj >> 2) & 1u, a.status);
                         ok = __all_sync(0xffffffffu, ok);
                         if (ok) {
                             tc_fence_after();
