@@ -528,16 +528,19 @@ score_pool_kernel(int Hk, int max_sent, int max_cap, const int32_t* cap, const i
 }
 
 // ---------------------------------------------------------------------------------------
-// Gram passes on the tensor cores.  CTA = 128 sentences i of one slab against all j in blocks of 128.
+// Gram passes on the tensor cores.  Work item = 128 sentences i of one slab against all j in blocks of 128;
+// persistent CTAs take the items round-robin, so barriers, tensor memory and descriptors are set up once and
+// the j-block ring keeps streaming from one item into the next.
 // ---------------------------------------------------------------------------------------
 struct GramCtl {
-    uint64_t afull, bfull[2], bempty[2], tfull[2], tempty[2];
+    uint64_t afull, aempty, bfull[2], bempty[2], tfull[2], tempty[2];
     uint32_t tmem_base;
     int abort_flag;
+    uint32_t wsum[8];
     float invz[2][128];
 };
 constexpr int kGramThreads = 6 * 32;
-constexpr size_t kGramSmem = 1024 + 6 * size_t(kOpBytes) + sizeof(GramCtl);
+static size_t gram_smem_bytes(int slabs) { return 1024 + 6 * size_t(kOpBytes) + sizeof(GramCtl) + size_t(slabs + 1) * 4; }
 
 __device__ __forceinline__ bool gram_wait(GramCtl* ctl, uint64_t* bar, uint32_t parity, uint32_t* status) {
     if (mbar_try_wait(bar, parity)) return true;
@@ -555,24 +558,22 @@ __device__ __forceinline__ bool gram_wait(GramCtl* ctl, uint64_t* bar, uint32_t 
 
 template <int kPass>
 __global__ void __launch_bounds__(kGramThreads, 1)
-score_gram_kernel(const __grid_constant__ CUtensorMap mapHi, const __grid_constant__ CUtensorMap mapLo, int max_sent,
-                  const int32_t* n_sent, float sigma, float tau, float* sc_z, const float* sent_imp, float* sent_red,
-                  float* sent_lam, float* sent_score, uint32_t* status) {
+score_gram_kernel(const __grid_constant__ CUtensorMap mapHi, const __grid_constant__ CUtensorMap mapLo, int n_slabs,
+                  int max_sent, const int32_t* n_sent, float sigma, float tau, float* sc_z, const float* sent_imp,
+                  float* sent_red, float* sent_lam, float* sent_score, uint32_t* status) {
     extern __shared__ uint8_t gram_smem_raw[];
-    const int slab = blockIdx.y;
-    const int S = min(max(n_sent[slab], 0), max_sent);
-    const int i0 = blockIdx.x * 128;
-    if (i0 >= S) return;
     const uint32_t raw = smem_u32(gram_smem_raw);
     uint8_t* At = gram_smem_raw + (((raw + 1023u) & ~1023u) - raw);              // hi, lo of the i block
     uint8_t* Bt = At + 2 * kOpBytes;                                             // 2 stages x (hi, lo) of a j block
     GramCtl* ctl = reinterpret_cast<GramCtl*>(Bt + 4 * kOpBytes);
+    int* ipref = reinterpret_cast<int*>(ctl + 1);                                // [n_slabs + 1] prefix of i blocks
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int NJ = (S + 127) >> 7;
-    const int rowbase = slab * max_sent;
+    const int G = gridDim.x, cta = blockIdx.x;
+    auto sent_of = [&](int s) { return min(max(n_sent[s], 0), max_sent); };
 
     if (tid == 0) {
         mbar_init(&ctl->afull, 1);
+        mbar_init(&ctl->aempty, 1);
         for (int s = 0; s < 2; ++s) {
             mbar_init(&ctl->bfull[s], 1);
             mbar_init(&ctl->bempty[s], 1);
@@ -585,123 +586,173 @@ score_gram_kernel(const __grid_constant__ CUtensorMap mapHi, const __grid_consta
         tmap_prefetch(&mapLo);
     }
     if (warp == 1) tmem_alloc(&ctl->tmem_base, 256);
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
+    {   // prefix of i blocks over slabs (block scan; every thread owns a contiguous block of slabs)
+        const int per = (n_slabs + kGramThreads - 1) / kGramThreads;
+        const int s0 = min(tid * per, n_slabs), s1 = min(s0 + per, n_slabs);
+        uint32_t local = 0;
+        for (int s = s0; s < s1; ++s) local += uint32_t((sent_of(s) + 127) >> 7);
+        uint32_t inc = local;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const uint32_t x = __shfl_up_sync(0xffffffffu, inc, d);
+            if (lane >= d) inc += x;
+        }
+        if (lane == 31) ctl->wsum[warp] = inc;
+        tc_fence_before();
+        __syncthreads();                                 // also publishes barrier inits and the tmem address
+        tc_fence_after();
+        uint32_t base = 0;
+        for (int w = 0; w < warp; ++w) base += ctl->wsum[w];
+        uint32_t run = base + inc - local;
+        for (int s = s0; s < s1; ++s) {
+            ipref[s] = int(run);
+            run += uint32_t((sent_of(s) + 127) >> 7);
+        }
+        if (tid == kGramThreads - 1) ipref[n_slabs] = int(run);
+        __syncthreads();
+    }
     const uint32_t tmem_base = ctl->tmem_base;
+    const int n_items = ipref[n_slabs];
 
     if (warp == 0) {
         if (lane == 0) {
-            mbar_expect_tx(&ctl->afull, 2 * kOpBytes);
-            tma_load_2d(At, &mapHi, 0, rowbase + i0, &ctl->afull);
-            tma_load_2d(At + kOpHalfBytes, &mapHi, 64, rowbase + i0, &ctl->afull);
-            tma_load_2d(At + kOpBytes, &mapLo, 0, rowbase + i0, &ctl->afull);
-            tma_load_2d(At + kOpBytes + kOpHalfBytes, &mapLo, 64, rowbase + i0, &ctl->afull);
             bool ok = true;
-            for (int jb = 0; jb < NJ && ok; ++jb) {
-                const int s = jb & 1;
-                if (jb >= 2) ok = gram_wait(ctl, &ctl->bempty[s], uint32_t((jb >> 1) - 1) & 1u, status);
+            int slab = 0;
+            uint32_t bc = 0, ic = 0;                                // j blocks and items issued so far
+            for (int item = cta; item < n_items && ok; item += G, ++ic) {
+                while (ipref[slab + 1] <= item) ++slab;
+                const int S = sent_of(slab), NJ = (S + 127) >> 7, rowbase = slab * max_sent;
+                const int i0 = (item - ipref[slab]) * 128;
+                if (ic > 0) ok = gram_wait(ctl, &ctl->aempty, (ic - 1) & 1u, status);
                 if (!ok) break;
-                uint8_t* dst = Bt + size_t(s) * 2 * kOpBytes;
-                mbar_expect_tx(&ctl->bfull[s], 2 * kOpBytes);
-                tma_load_2d(dst, &mapHi, 0, rowbase + jb * 128, &ctl->bfull[s]);
-                tma_load_2d(dst + kOpHalfBytes, &mapHi, 64, rowbase + jb * 128, &ctl->bfull[s]);
-                tma_load_2d(dst + kOpBytes, &mapLo, 0, rowbase + jb * 128, &ctl->bfull[s]);
-                tma_load_2d(dst + kOpBytes + kOpHalfBytes, &mapLo, 64, rowbase + jb * 128, &ctl->bfull[s]);
+                mbar_expect_tx(&ctl->afull, 2 * kOpBytes);
+                tma_load_2d(At, &mapHi, 0, rowbase + i0, &ctl->afull);
+                tma_load_2d(At + kOpHalfBytes, &mapHi, 64, rowbase + i0, &ctl->afull);
+                tma_load_2d(At + kOpBytes, &mapLo, 0, rowbase + i0, &ctl->afull);
+                tma_load_2d(At + kOpBytes + kOpHalfBytes, &mapLo, 64, rowbase + i0, &ctl->afull);
+                for (int jb = 0; jb < NJ && ok; ++jb, ++bc) {
+                    const int s = bc & 1;
+                    if (bc >= 2) ok = gram_wait(ctl, &ctl->bempty[s], ((bc >> 1) - 1) & 1u, status);
+                    if (!ok) break;
+                    uint8_t* dst = Bt + size_t(s) * 2 * kOpBytes;
+                    mbar_expect_tx(&ctl->bfull[s], 2 * kOpBytes);
+                    tma_load_2d(dst, &mapHi, 0, rowbase + jb * 128, &ctl->bfull[s]);
+                    tma_load_2d(dst + kOpHalfBytes, &mapHi, 64, rowbase + jb * 128, &ctl->bfull[s]);
+                    tma_load_2d(dst + kOpBytes, &mapLo, 0, rowbase + jb * 128, &ctl->bfull[s]);
+                    tma_load_2d(dst + kOpBytes + kOpHalfBytes, &mapLo, 64, rowbase + jb * 128, &ctl->bfull[s]);
+                }
             }
             if (!ok) {
-                mbar_wait(&ctl->afull, 0u, 1u << 16);
+                mbar_wait(&ctl->afull, 0u, 1u << 16); mbar_wait(&ctl->afull, 1u, 1u << 16);
                 for (int s = 0; s < 2; ++s) { mbar_wait(&ctl->bfull[s], 0u, 1u << 16); mbar_wait(&ctl->bfull[s], 1u, 1u << 16); }
             }
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            bool ok = gram_wait(ctl, &ctl->afull, 0u, status);
+            bool ok = true;
+            int slab = 0;
+            uint32_t bc = 0, ic = 0;
             const uint32_t a_hi = smem_u32(At), a_lo = smem_u32(At + kOpBytes);
-            for (int jb = 0; jb < NJ && ok; ++jb) {
-                const int s = jb & 1;
-                ok = gram_wait(ctl, &ctl->bfull[s], uint32_t(jb >> 1) & 1u, status);
-                if (ok && jb >= 2) ok = gram_wait(ctl, &ctl->tempty[s], uint32_t((jb >> 1) - 1) & 1u, status);
-                if (!ok) break;
-                tc_fence_after();
-                const uint32_t b_hi = smem_u32(Bt + size_t(s) * 2 * kOpBytes), b_lo = b_hi + kOpBytes;
-                const uint32_t d = tmem_base + s * 128;
-                umma_tile_128x128x128(d, a_hi, b_hi, false);
-                umma_tile_128x128x128(d, a_hi, b_lo, true);
-                umma_tile_128x128x128(d, a_lo, b_hi, true);
-                umma_commit(&ctl->tfull[s]);
-                umma_commit(&ctl->bempty[s]);
+            for (int item = cta; item < n_items && ok; item += G, ++ic) {
+                while (ipref[slab + 1] <= item) ++slab;
+                const int NJ = (sent_of(slab) + 127) >> 7;
+                ok = gram_wait(ctl, &ctl->afull, ic & 1u, status);
+                for (int jb = 0; jb < NJ && ok; ++jb, ++bc) {
+                    const int s = bc & 1;
+                    ok = gram_wait(ctl, &ctl->bfull[s], (bc >> 1) & 1u, status);
+                    if (ok && bc >= 2) ok = gram_wait(ctl, &ctl->tempty[s], ((bc >> 1) - 1) & 1u, status);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t b_hi = smem_u32(Bt + size_t(s) * 2 * kOpBytes), b_lo = b_hi + kOpBytes;
+                    const uint32_t d = tmem_base + s * 128;
+                    umma_tile_128x128x128(d, a_hi, b_hi, false);
+                    umma_tile_128x128x128(d, a_hi, b_lo, true);
+                    umma_tile_128x128x128(d, a_lo, b_hi, true);
+                    umma_commit(&ctl->tfull[s]);
+                    umma_commit(&ctl->bempty[s]);
+                }
+                if (ok) umma_commit(&ctl->aempty);                   // every MMA that reads this i block has completed
             }
         }
     } else {
         const int quarter = warp & 3, wt = tid - 64;
-        const int i = i0 + quarter * 32 + lane;
         const uint32_t lane_addr = tmem_base + (uint32_t(quarter * 32) << 16);
-        float accum = 0.f, mx = -INFINITY;
         bool ok = true;
-        for (int jb = 0; jb < NJ && ok; ++jb) {
-            const int s = jb & 1, j0 = jb * 128;
-            if (kPass == 2) {
-                const int j = j0 + wt;
-                const float z = (j < S) ? sc_z[size_t(rowbase) + j] : 1.f;
-                ctl->invz[s][wt] = (z > 0.f) ? 1.f / z : 0.f;
-                named_bar_sync(1, 128);
-            }
-            ok = gram_wait(ctl, &ctl->tfull[s], uint32_t(jb >> 1) & 1u, status);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            tc_fence_after();
-            const bool interior = (j0 + 128 <= S) && (j0 != i0);
+        int slab = 0;
+        uint32_t bc = 0;
+        for (int item = cta; item < n_items; item += G) {
+            while (ipref[slab + 1] <= item) ++slab;
+            const int S = sent_of(slab), NJ = (S + 127) >> 7, rowbase = slab * max_sent;
+            const int i0 = (item - ipref[slab]) * 128;
+            const int i = i0 + quarter * 32 + lane;
+            float accum = 0.f, mx = -INFINITY;
+            for (int jb = 0; jb < NJ; ++jb, ++bc) {
+                const int s = bc & 1, j0 = jb * 128;
+                if (kPass == 2) {
+                    const int j = j0 + wt;
+                    const float z = (j < S) ? sc_z[size_t(rowbase) + j] : 1.f;
+                    ctl->invz[s][wt] = (z > 0.f) ? 1.f / z : 0.f;
+                    named_bar_sync(1, 128);
+                }
+                if (ok) {
+                    ok = gram_wait(ctl, &ctl->tfull[s], (bc >> 1) & 1u, status);
+                    ok = __all_sync(0xffffffffu, ok);
+                }
+                if (!ok) continue;                               // keeps the barrier pattern uniform
+                tc_fence_after();
+                const bool interior = (j0 + 128 <= S) && (j0 != i0);
+#pragma unroll 1
+                for (int ch = 0; ch < 4; ++ch) {
+                    float v[32];
+                    tmem_ld32(lane_addr + s * 128 + ch * 32, v);
+                    const float* iz = ctl->invz[s] + ch * 32;
+                    if (interior) {
+                        float e0 = 0.f, e1 = 0.f;
 #pragma unroll
-            for (int ch = 0; ch < 4; ++ch) {
-                float v[32];
-                tmem_ld32(lane_addr + s * 128 + ch * 32, v);
-                if (interior) {
-                    float e0 = 0.f, e1 = 0.f;
-#pragma unroll
-                    for (int jj = 0; jj < 32; jj += 2) {
-                        if (kPass == 1) {
-                            e0 += ex2f(v[jj] * kLog2e);
-                            e1 += ex2f(v[jj + 1] * kLog2e);
-                        } else {
-                            e0 = fmaf(ex2f(v[jj] * kLog2e), ctl->invz[s][ch * 32 + jj], e0);
-                            e1 = fmaf(ex2f(v[jj + 1] * kLog2e), ctl->invz[s][ch * 32 + jj + 1], e1);
-                        }
-                    }
-                    accum += e0 + e1;
-                    if (kPass == 1 && j0 > i0) {
-#pragma unroll
-                        for (int jj = 0; jj < 32; ++jj) mx = fmaxf(mx, v[jj]);
-                    }
-                } else {
-#pragma unroll
-                    for (int jj = 0; jj < 32; ++jj) {
-                        const int j = j0 + ch * 32 + jj;
-                        if (j < S && j != i) {
-                            const float e = ex2f(v[jj] * kLog2e);
+                        for (int jj = 0; jj < 32; jj += 2) {
                             if (kPass == 1) {
-                                accum += e;
-                                if (j > i) mx = fmaxf(mx, v[jj]);
+                                e0 += ex2f(v[jj] * kLog2e);
+                                e1 += ex2f(v[jj + 1] * kLog2e);
                             } else {
-                                accum = fmaf(e, ctl->invz[s][ch * 32 + jj], accum);
+                                e0 = fmaf(ex2f(v[jj] * kLog2e), iz[jj], e0);
+                                e1 = fmaf(ex2f(v[jj + 1] * kLog2e), iz[jj + 1], e1);
+                            }
+                        }
+                        accum += e0 + e1;
+                        if (kPass == 1 && j0 > i0) {
+#pragma unroll
+                            for (int jj = 0; jj < 32; ++jj) mx = fmaxf(mx, v[jj]);
+                        }
+                    } else {
+#pragma unroll
+                        for (int jj = 0; jj < 32; ++jj) {
+                            const int j = j0 + ch * 32 + jj;
+                            if (j < S && j != i) {
+                                const float e = ex2f(v[jj] * kLog2e);
+                                if (kPass == 1) {
+                                    accum += e;
+                                    if (j > i) mx = fmaxf(mx, v[jj]);
+                                } else {
+                                    accum = fmaf(e, iz[jj], accum);
+                                }
                             }
                         }
                     }
                 }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&ctl->tempty[s]);
             }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&ctl->tempty[s]);
-        }
-        if (ok && i < S) {
-            const size_t o = size_t(rowbase) + i;
-            if (kPass == 1) {
-                sc_z[o] = accum;
-                sent_lam[o] = (mx > tau) ? mx : 0.f;
-            } else {
-                const float red = accum / float(S);
-                sent_red[o] = red;
-                sent_score[o] = sigma * sent_imp[o] - (1.f - sigma) * red - sent_lam[o];
+            if (ok && i < S) {
+                const size_t o = size_t(rowbase) + i;
+                if (kPass == 1) {
+                    sc_z[o] = accum;
+                    sent_lam[o] = (mx > tau) ? mx : 0.f;
+                } else {
+                    const float red = accum / float(S);
+                    sent_red[o] = red;
+                    sent_score[o] = sigma * sent_imp[o] - (1.f - sigma) * red - sent_lam[o];
+                }
             }
         }
     }
@@ -794,16 +845,19 @@ extern "C" int skipkv_score(const skipkv_shape* shape, const skipkv_params* para
         SKIPKV_CUDA(cudaGetLastError());
     }
     {
-        dim3 ggrid((shape->max_sent + 127) / 128, L.slabs);
-        SKIPKV_CUDA(cudaFuncSetAttribute(score_gram_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kGramSmem)));
-        SKIPKV_CUDA(cudaFuncSetAttribute(score_gram_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kGramSmem)));
-        score_gram_kernel<1><<<ggrid, kGramThreads, kGramSmem, st>>>(mapHi, mapLo, shape->max_sent, n_sent, params->sigma,
-                                                                    params->tau, sc_z, sent_imp, sent_red, sent_lam,
-                                                                    sent_score, status);
+        const size_t gsmem = gram_smem_bytes(L.slabs);
+        if (gsmem > 227 * 1024) return SKIPKV_ERR_UNSUPPORTED;
+        const long long max_items = (long long)L.slabs * ((shape->max_sent + 127) / 128);
+        const int ggrid = int(max_items < (long long)grid ? max_items : (long long)grid);
+        SKIPKV_CUDA(cudaFuncSetAttribute(score_gram_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(gsmem)));
+        SKIPKV_CUDA(cudaFuncSetAttribute(score_gram_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(gsmem)));
+        score_gram_kernel<1><<<ggrid, kGramThreads, gsmem, st>>>(mapHi, mapLo, L.slabs, shape->max_sent, n_sent, params->sigma,
+                                                                 params->tau, sc_z, sent_imp, sent_red, sent_lam, sent_score,
+                                                                 status);
         SKIPKV_CUDA(cudaGetLastError());
-        score_gram_kernel<2><<<ggrid, kGramThreads, kGramSmem, st>>>(mapHi, mapLo, shape->max_sent, n_sent, params->sigma,
-                                                                    params->tau, sc_z, sent_imp, sent_red, sent_lam,
-                                                                    sent_score, status);
+        score_gram_kernel<2><<<ggrid, kGramThreads, gsmem, st>>>(mapHi, mapLo, L.slabs, shape->max_sent, n_sent, params->sigma,
+                                                                 params->tau, sc_z, sent_imp, sent_red, sent_lam, sent_score,
+                                                                 status);
         SKIPKV_CUDA(cudaGetLastError());
     }
     return SKIPKV_OK;
