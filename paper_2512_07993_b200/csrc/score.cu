@@ -33,9 +33,10 @@ constexpr int kAccBufs = 4;             // tensor-memory accumulators of 128 col
 constexpr int kMaxRB = 4;               // query blocks per group
 constexpr int kSwMaxStages = 6;
 constexpr int kSw1Groups = 4;           // epilogue warpgroups of sweep 1
-constexpr int kSw2Groups = 3;           // epilogue warpgroups of sweep 2 (plus one pooling warpgroup)
+constexpr int kSw2Groups = 2;           // epilogue warpgroups of sweep 2
+constexpr int kPoolWarps = 8;           // pooling warps of sweep 2: warp p sums the key rows of tiles p, p + 8, ...
 constexpr int kSw1Threads = (2 + 4 * kSw1Groups) * 32;        // TMA warp, MMA warp, epilogue warps
-constexpr int kSw2Threads = (2 + 4 * kSw2Groups + 4) * 32;    // + 4 pooling warps
+constexpr int kSw2Threads = (2 + 4 * kSw2Groups + kPoolWarps) * 32;
 constexpr float kLog2e = 1.4426950408889634f;
 
 __device__ __forceinline__ float ex2f(float x) {
@@ -53,6 +54,7 @@ struct SweepCtl {                       // barriers and small shared state, afte
     uint64_t tfull[4][4], tempty[kAccBufs];
     uint32_t tmem_base;
     int abort_flag;
+    int landed;                         // sweep 2: tiles whose copy has completed (a monotone count for the pooling warps)
     uint32_t wsum[16];
     alignas(16) float neg_lse[kSw2Groups][kMaxRB * 128];   // sweep 2: one copy per epilogue warpgroup (read as float4)
 };
@@ -60,6 +62,7 @@ static_assert(offsetof(SweepCtl, neg_lse) % 16 == 0, "neg_lse is read with 16-by
 
 struct SweepArgs {
     int Hq, Hk, window, n_slabs, max_cap, max_sent, RB, WB, stages;
+    int so_smem;                        // sweep 2: sentence offsets and per-tile first sentences are staged in shared memory
     const int64_t* slab_off;
     const int32_t* cap;
     const int32_t* kv_len;
@@ -169,7 +172,7 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_consta
     if (tid == 0) {
         for (int s = 0; s < kSwMaxStages; ++s) {
             mbar_init(&ctl->full[s], 1);
-            mbar_init(&ctl->empty[s], kSweep == 1 ? 1 : 5);      // MMA commit (+ 4 pooling warps)
+            mbar_init(&ctl->empty[s], kSweep == 1 ? 1 : 2);      // MMA commit (+ the tile's pooling warp)
         }
         mbar_init(&ctl->qfull, 1);
         mbar_init(&ctl->qempty, 1);
@@ -177,6 +180,7 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_consta
         for (int g = 0; g < 4; ++g)
             for (int j = 0; j < 4; ++j) mbar_init(&ctl->tfull[g][j], 1);
         ctl->abort_flag = 0;
+        ctl->landed = 0;
         mbar_fence_init();
         tmap_prefetch(&mapK);
         tmap_prefetch(&mapQ);
@@ -278,6 +282,10 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_consta
                 }
                 ok = ctl_wait(ctl, &ctl->full[stage], lap & 1u, a.status);
                 if (!ok) break;
+                if (kSweep == 2) {                       // pooling warps skip tiles, so they follow a count, not barrier phases
+                    __threadfence_block();
+                    *reinterpret_cast<volatile int*>(&ctl->landed) = t - t_begin + 1;
+                }
                 const uint32_t k_smem = smem_u32(tiles + size_t(stage) * kOpBytes);
                 for (int k = 0; k < RB && ok; ++k, ++it) {
                     const int buf = it & (kAccBufs - 1), use = it / kAccBufs;
@@ -398,78 +406,110 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_consta
         }
     } else if (kSweep == 2) {
         // ------------------------------------------------------------------ pooling warps: per-sentence sums of key rows
-        // warp pw owns rows [32 pw, 32 pw + 32) of every tile; a lane owns 4 channels (8 bytes) of a row
+        // Loads from shared memory wait several hundred cycles here (the tensor core streams its operands from the
+        // same memory), so the work is arranged for few dependent steps: pooling warp p takes whole tiles
+        // (p, p + 8, ...), which gives it eight tile periods per tile; the sentence of a tile's first token comes
+        // from a table built once per slab; the starts of the following sentences are fetched in one access; rows
+        // are loaded sixteen at a time.  A lane owns 4 channels (8 bytes) of every row.
         const int pw = warp - (2 + 4 * kGroups);
+        const int ptid = tid - (2 + 4 * kGroups) * 32;                 // thread index among the pooling warps
         const int half = lane >> 4, chunk = (lane & 15) >> 1, sub = (lane & 1) * 8;
         const int ch0 = half * 64 + (lane & 15) * 4;                   // first channel of this lane
-        int swz[8];                                                    // byte offset of this lane's chunk in row i of 8
-#pragma unroll
-        for (int i = 0; i < 8; ++i) swz[i] = i * 128 + ((chunk ^ i) << 4);
-        int slab = slab0, S = 0, N = 0, cur = -1;
+        int32_t* so_stage = reinterpret_cast<int32_t*>(pref + n_slabs + 1);       // [max_sent + 1]
+        int32_t* tfirst = so_stage + (a.max_sent + 1);                            // [tiles of the slab]
+        int slab = slab0, S = 0, N = 0;
         const int32_t* so = a.sent_off;
         bool ok = true, have = false;
-        for (int tl = 0; tl < ntl && ok; ++tl) {
+        for (int tl = 0; tl < ntl; ++tl) {
             const int t = t_begin + tl, stage = tl % a.stages;
-            ok = ctl_wait(ctl, &ctl->full[stage], uint32_t(tl / a.stages) & 1u, a.status);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
             if (!have || pref[slab + 1] <= t) {
+                // new slab (all pooling warps get here at the same tile): stage its sentence offsets and the
+                // sentence of every tile's first token; the first barrier ends the reads of the old tables
                 while (pref[slab + 1] <= t) ++slab;
                 have = true;
                 S = min(max(a.n_sent[slab], 0), a.max_sent);
                 so = a.sent_off + size_t(slab) * (a.max_sent + 1);
                 N = live(slab);
-                cur = -1;
+                if (a.so_smem) {
+                    named_bar_sync(8, kPoolWarps * 32);
+                    for (int i = ptid; i <= S; i += kPoolWarps * 32) so_stage[i] = so[i];
+                    named_bar_sync(8, kPoolWarps * 32);
+                    so = so_stage;
+                    const int nt = (N + 127) >> 7;
+                    for (int j = ptid; j < nt; j += kPoolWarps * 32) {
+                        int lo = 0, hi = max(S - 1, 0);
+                        while (lo < hi) {
+                            const int mid = (lo + hi + 1) >> 1;
+                            if (so[mid] <= j * 128) lo = mid; else hi = mid - 1;
+                        }
+                        tfirst[j] = lo;
+                    }
+                    named_bar_sync(8, kPoolWarps * 32);
+                }
             }
+            if ((tl % kPoolWarps) != pw) continue;              // another pooling warp's tile
+            if (ok) {                                           // wait (bounded) until the tile's copy has landed
+                uint32_t spins = 0;
+                while (*reinterpret_cast<volatile int*>(&ctl->landed) <= tl) {
+                    if (*reinterpret_cast<volatile int*>(&ctl->abort_flag) || ++spins > (1u << 22)) { ok = false; break; }
+                    __nanosleep(64);
+                }
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok && lane == 0) {
+                    atomicOr(a.status, SKIPKV_STATUS_COPY_TIMEOUT);
+                    *reinterpret_cast<volatile int*>(&ctl->abort_flag) = 1;
+                }
+                __threadfence_block();
+            }
+            if (!ok) continue;
             const int tok0 = (t - pref[slab]) * 128;
-            const int r_lo = pw * 32, r_hi = min(r_lo + 32, N - tok0);
-            if (S > 0 && r_lo < r_hi) {
-                const int tk = tok0 + r_lo;
-                if (cur < 0) {
+            const int nrows = min(128, N - tok0);
+            if (S > 0 && nrows > 0) {
+                int cur;
+                if (a.so_smem) {
+                    cur = tfirst[t - pref[slab]];
+                } else {
                     int lo = 0, hi = S - 1;
                     while (lo < hi) {
                         const int mid = (lo + hi + 1) >> 1;
-                        if (so[mid] <= tk) lo = mid; else hi = mid - 1;
+                        if (so[mid] <= tok0) lo = mid; else hi = mid - 1;
                     }
                     cur = lo;
-                } else {
-                    while (cur + 1 < S && so[cur + 1] <= tk) ++cur;
                 }
+                // tile-relative starts of the next 32 sentences, one per lane (refilled if a tile has more)
+                int base = cur + 1;
+                int my = (base + lane < S) ? so[base + lane] - tok0 : 0x7fffffff;
                 const uint8_t* colbase = tiles + size_t(stage) * kOpBytes + half * kOpHalfBytes + sub;
-                auto ld = [&](int r) {
-                    return *reinterpret_cast<const uint2*>(colbase + r * 128 + ((chunk ^ (r & 7)) << 4));
-                };
-                int r = r_lo;
-                while (r < r_hi) {
-                    int e = r_hi;
-                    if (cur + 1 < S) e = min(e, so[cur + 1] - tok0);
+                float* dst = a.vsum + size_t(slab) * a.max_sent * kHeadDim + ch0;
+                int r = 0;
+                while (r < nrows) {
+                    // piece [r, e): rows of sentence `cur`
+                    int e = nrows;
+                    if (cur + 1 < S) {
+                        if (cur + 1 - base >= 32) { base = cur + 1; my = (base + lane < S) ? so[base + lane] - tok0 : 0x7fffffff; }
+                        e = min(e, __shfl_sync(0xffffffffu, my, cur + 1 - base));
+                    }
                     if (e > r) {
                         float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-                        for (; (r & 7) && r < e; ++r) {          // up to a swizzle-period boundary
-                            const uint2 u = ld(r);
-                            a0 += bf16lo(u.x); a1 += bf16hi(u.x);
-                            a2 += bf16lo(u.y); a3 += bf16hi(u.y);
-                        }
-                        for (; r + 8 <= e; r += 8) {             // r % 8 == 0: the offsets are the precomputed ones
-                            const uint8_t* rp = colbase + r * 128;
-                            uint2 u[8];
+#pragma unroll 1
+                        for (int rb = r; rb < e; rb += 16) {    // sixteen rows in flight; rows past the piece load as zero
+                            uint2 u[16];
 #pragma unroll
-                            for (int i = 0; i < 8; ++i) u[i] = *reinterpret_cast<const uint2*>(rp + swz[i]);
+                            for (int i = 0; i < 16; ++i) {
+                                const int rr = rb + i;
+                                u[i] = (rr < e) ? *reinterpret_cast<const uint2*>(colbase + rr * 128 + ((chunk ^ (rr & 7)) << 4))
+                                                : make_uint2(0u, 0u);
+                            }
 #pragma unroll
-                            for (int i = 0; i < 8; ++i) {
+                            for (int i = 0; i < 16; ++i) {
                                 a0 += bf16lo(u[i].x); a1 += bf16hi(u[i].x);
                                 a2 += bf16lo(u[i].y); a3 += bf16hi(u[i].y);
                             }
                         }
-                        for (; r < e; ++r) {
-                            const uint2 u = ld(r);
-                            a0 += bf16lo(u.x); a1 += bf16hi(u.x);
-                            a2 += bf16lo(u.y); a3 += bf16hi(u.y);
-                        }
-                        atomicAdd(reinterpret_cast<float4*>(a.vsum + (size_t(slab) * a.max_sent + cur) * kHeadDim + ch0),
-                                  make_float4(a0, a1, a2, a3));
+                        atomicAdd(reinterpret_cast<float4*>(dst + size_t(cur) * kHeadDim), make_float4(a0, a1, a2, a3));
+                        r = e;
                     }
-                    if (r < r_hi) ++cur;                     // the piece ended on a sentence boundary
+                    if (r < nrows) ++cur;                       // the piece ended on a sentence boundary
                 }
             }
             __syncwarp();
@@ -813,28 +853,36 @@ extern "C" int skipkv_score(const skipkv_shape* shape, const skipkv_params* para
     a.slab_off = shape->slab_off; a.cap = shape->cap; a.kv_len = kv_len; a.sent_off = sent_off; a.n_sent = n_sent;
     a.sc_part = reinterpret_cast<float2*>(w + L.sc_part);
     a.tok_imp_user = tok_imp; a.tok_imp_ws = sc_tok; a.vsum = vsum; a.status = status;
-    const size_t fixed = 1024 + size_t(a.RB) * kOpBytes + sizeof(SweepCtl) + size_t(L.slabs + 1) * 4;
     const size_t max_smem = 227 * 1024;
-    if (fixed + kOpBytes > max_smem) return SKIPKV_ERR_UNSUPPORTED;
-    int stages = int((max_smem - fixed) / kOpBytes);
-    if (stages > kSwMaxStages) stages = kSwMaxStages;
-    a.stages = stages;
-    const size_t smem = fixed + size_t(stages) * kOpBytes;
+    const size_t fixed1 = 1024 + size_t(a.RB) * kOpBytes + sizeof(SweepCtl) + size_t(L.slabs + 1) * 4;
+    if (fixed1 + kOpBytes > max_smem) return SKIPKV_ERR_UNSUPPORTED;
+    SweepArgs a1 = a, a2 = a;
+    a1.so_smem = 0;
+    a1.stages = int((max_smem - fixed1) / kOpBytes);
+    if (a1.stages > kSwMaxStages) a1.stages = kSwMaxStages;
+    // sweep 2 also stages the current slab's sentence offsets and one sentence index per tile of the slab, when
+    // that leaves at least two tile stages (otherwise its pooling warps read the table from global memory)
+    const size_t tab_bytes = (size_t(shape->max_sent) + 1 + size_t((shape->max_cap + 127) / 128)) * 4;
+    a2.so_smem = (fixed1 + tab_bytes + 2 * kOpBytes <= max_smem) ? 1 : 0;
+    const size_t fixed2 = fixed1 + (a2.so_smem ? tab_bytes : 0);
+    a2.stages = int((max_smem - fixed2) / kOpBytes);
+    if (a2.stages > kSwMaxStages) a2.stages = kSwMaxStages;
+    const size_t smem1 = fixed1 + size_t(a1.stages) * kOpBytes, smem2 = fixed2 + size_t(a2.stages) * kOpBytes;
     int grid = num_sms();
     if (grid > L.dec_max_ctas) grid = L.dec_max_ctas;
 
     SKIPKV_CUDA(cudaMemsetAsync(vsum, 0, size_t(L.slabs) * shape->max_sent * kHeadDim * 4, st));
-    if (int rc = launch_sweep<1, 1>(mapK, mapQ, a, grid, smem, st)) return rc;
+    if (int rc = launch_sweep<1, 1>(mapK, mapQ, a1, grid, smem1, st)) return rc;
     int rc = SKIPKV_ERR_UNSUPPORTED;
     switch (n) {
-        case 1: rc = launch_sweep<2, 1>(mapK, mapQ, a, grid, smem, st); break;
-        case 2: rc = launch_sweep<2, 2>(mapK, mapQ, a, grid, smem, st); break;
-        case 3: rc = launch_sweep<2, 3>(mapK, mapQ, a, grid, smem, st); break;
-        case 4: rc = launch_sweep<2, 4>(mapK, mapQ, a, grid, smem, st); break;
-        case 5: rc = launch_sweep<2, 5>(mapK, mapQ, a, grid, smem, st); break;
-        case 6: rc = launch_sweep<2, 6>(mapK, mapQ, a, grid, smem, st); break;
-        case 7: rc = launch_sweep<2, 7>(mapK, mapQ, a, grid, smem, st); break;
-        case 8: rc = launch_sweep<2, 8>(mapK, mapQ, a, grid, smem, st); break;
+        case 1: rc = launch_sweep<2, 1>(mapK, mapQ, a2, grid, smem2, st); break;
+        case 2: rc = launch_sweep<2, 2>(mapK, mapQ, a2, grid, smem2, st); break;
+        case 3: rc = launch_sweep<2, 3>(mapK, mapQ, a2, grid, smem2, st); break;
+        case 4: rc = launch_sweep<2, 4>(mapK, mapQ, a2, grid, smem2, st); break;
+        case 5: rc = launch_sweep<2, 5>(mapK, mapQ, a2, grid, smem2, st); break;
+        case 6: rc = launch_sweep<2, 6>(mapK, mapQ, a2, grid, smem2, st); break;
+        case 7: rc = launch_sweep<2, 7>(mapK, mapQ, a2, grid, smem2, st); break;
+        case 8: rc = launch_sweep<2, 8>(mapK, mapQ, a2, grid, smem2, st); break;
         default: break;
     }
     if (rc) return rc;
