@@ -229,6 +229,13 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_consta
     const float scale = kLog2e * rsqrtf(float(kHeadDim));
     const int n = a.Hq / Hk;
 
+    if (kSweep == 1 && warp < 2 && lane != 0) {
+        // the 62 otherwise idle lanes of the TMA and MMA warps clear the per-sentence key sums that sweep 2 accumulates
+        const size_t total = size_t(n_slabs) * a.max_sent * (kHeadDim / 4);        // float4 words
+        const size_t per = (total + G - 1) / G, w0 = min(size_t(cta) * per, total), w1 = min(w0 + per, total);
+        float4* v4 = reinterpret_cast<float4*>(a.vsum);
+        for (size_t i = w0 + size_t(warp * 31 + lane - 1); i < w1; i += 62) v4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0 && ntl > 0) {
@@ -871,7 +878,6 @@ extern "C" int skipkv_score(const skipkv_shape* shape, const skipkv_params* para
     int grid = num_sms();
     if (grid > L.dec_max_ctas) grid = L.dec_max_ctas;
 
-    SKIPKV_CUDA(cudaMemsetAsync(vsum, 0, size_t(L.slabs) * shape->max_sent * kHeadDim * 4, st));
     if (int rc = launch_sweep<1, 1>(mapK, mapQ, a1, grid, smem1, st)) return rc;
     int rc = SKIPKV_ERR_UNSUPPORTED;
     switch (n) {

@@ -87,18 +87,18 @@ select_kernel(int max_sent, int P, int budget, int protect_tail, const float* se
         flags[i] = 0;
     }
     __syncthreads();
-    // bitonic sort, ascending
+    // bitonic sort, ascending.  Thread p of a pass owns the compare-exchange pair (i, i | j) with
+    // i = ((p & ~(j-1)) << 1) | (p & (j-1)).  For j <= 32 the 32 pairs of a warp stay inside the warp's own
+    // 64-key block, so those steps only need a warp barrier; a block barrier separates them from the wider steps.
     for (int k = 2; k <= P; k <<= 1) {
         for (int j = k >> 1; j > 0; j >>= 1) {
-            for (int i = tid; i < P; i += kSelThreads) {
-                const int l = i ^ j;
-                if (l > i) {
-                    const uint64_t a = keys[i], c = keys[l];
-                    const bool up = (i & k) == 0;
-                    if ((a > c) == up) { keys[i] = c; keys[l] = a; }
-                }
+            for (int p = tid; p < (P >> 1); p += kSelThreads) {
+                const int i = ((p & ~(j - 1)) << 1) | (p & (j - 1)), l = i | j;
+                const uint64_t a = keys[i], c = keys[l];
+                const bool up = (i & k) == 0;
+                if ((a > c) == up) { keys[i] = c; keys[l] = a; }
             }
-            __syncthreads();
+            if (j > 32 || j == 1) __syncthreads(); else __syncwarp();
         }
     }
     // running total of lengths in rank order; each thread owns a contiguous block of ranks
