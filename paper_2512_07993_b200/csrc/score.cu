@@ -34,7 +34,7 @@ constexpr int kMaxRB = 4;               // query blocks per group
 constexpr int kSwMaxStages = 6;
 constexpr int kSw1Groups = 4;           // epilogue warpgroups of sweep 1
 constexpr int kSw2Groups = 2;           // epilogue warpgroups of sweep 2
-constexpr int kPoolWarps = 8;           // pooling warps of sweep 2: warp p sums the key rows of tiles p, p + 8, ...
+constexpr int kPoolWarps = 8;           // pooling warps of sweep 2: warp p sums rows 32 (p & 3) .. +31 of the tiles of parity p >> 2
 constexpr int kSw1Threads = (2 + 4 * kSw1Groups) * 32;        // TMA warp, MMA warp, epilogue warps
 constexpr int kSw2Threads = (2 + 4 * kSw2Groups + kPoolWarps) * 32;
 constexpr float kLog2e = 1.4426950408889634f;
@@ -172,7 +172,7 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_consta
     if (tid == 0) {
         for (int s = 0; s < kSwMaxStages; ++s) {
             mbar_init(&ctl->full[s], 1);
-            mbar_init(&ctl->empty[s], kSweep == 1 ? 1 : 2);      // MMA commit (+ the tile's pooling warp)
+            mbar_init(&ctl->empty[s], kSweep == 1 ? 1 : 5);      // MMA commit (+ the tile's four pooling warps)
         }
         mbar_init(&ctl->qfull, 1);
         mbar_init(&ctl->qempty, 1);
@@ -414,10 +414,11 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_consta
     } else if (kSweep == 2) {
         // ------------------------------------------------------------------ pooling warps: per-sentence sums of key rows
         // Loads from shared memory wait several hundred cycles here (the tensor core streams its operands from the
-        // same memory), so the work is arranged for few dependent steps: pooling warp p takes whole tiles
-        // (p, p + 8, ...), which gives it eight tile periods per tile; the sentence of a tile's first token comes
-        // from a table built once per slab; the starts of the following sentences are fetched in one access; rows
-        // are loaded sixteen at a time.  A lane owns 4 channels (8 bytes) of every row.
+        // same memory), and a tile's stage is held until its pooling is done, so the work is arranged for few
+        // dependent steps and a short hold: four warps share a tile (32 rows each), two such groups alternate over
+        // the tiles; the sentence of a 32-row block's first token comes from a table built once per slab; the starts
+        // of the following sentences are fetched in one access; a warp's rows are loaded sixteen at a time.  A lane
+        // owns 4 channels (8 bytes) of every row.
         const int pw = warp - (2 + 4 * kGroups);
         const int ptid = tid - (2 + 4 * kGroups) * 32;                 // thread index among the pooling warps
         const int half = lane >> 4, chunk = (lane & 15) >> 1, sub = (lane & 1) * 8;
@@ -442,19 +443,19 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_consta
                     for (int i = ptid; i <= S; i += kPoolWarps * 32) so_stage[i] = so[i];
                     named_bar_sync(8, kPoolWarps * 32);
                     so = so_stage;
-                    const int nt = (N + 127) >> 7;
+                    const int nt = (N + 31) >> 5;                   // 32-row blocks of the slab
                     for (int j = ptid; j < nt; j += kPoolWarps * 32) {
                         int lo = 0, hi = max(S - 1, 0);
                         while (lo < hi) {
                             const int mid = (lo + hi + 1) >> 1;
-                            if (so[mid] <= j * 128) lo = mid; else hi = mid - 1;
+                            if (so[mid] <= j * 32) lo = mid; else hi = mid - 1;
                         }
                         tfirst[j] = lo;
                     }
                     named_bar_sync(8, kPoolWarps * 32);
                 }
             }
-            if ((tl % kPoolWarps) != pw) continue;              // another pooling warp's tile
+            if ((tl & 1) != (pw >> 2)) continue;                // the other group's tile
             if (ok) {                                           // wait (bounded) until the tile's copy has landed
                 uint32_t spins = 0;
                 while (*reinterpret_cast<volatile int*>(&ctl->landed) <= tl) {
@@ -469,12 +470,13 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_consta
                 __threadfence_block();
             }
             if (!ok) continue;
-            const int tok0 = (t - pref[slab]) * 128;
-            const int nrows = min(128, N - tok0);
+            const int row0 = (pw & 3) * 32;                     // this warp's rows of the tile: [row0, row0 + 32)
+            const int tok0 = (t - pref[slab]) * 128 + row0;
+            const int nrows = min(32, N - tok0);
             if (S > 0 && nrows > 0) {
                 int cur;
                 if (a.so_smem) {
-                    cur = tfirst[t - pref[slab]];
+                    cur = tfirst[tok0 >> 5];
                 } else {
                     int lo = 0, hi = S - 1;
                     while (lo < hi) {
@@ -486,7 +488,7 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_consta
                 // tile-relative starts of the next 32 sentences, one per lane (refilled if a tile has more)
                 int base = cur + 1;
                 int my = (base + lane < S) ? so[base + lane] - tok0 : 0x7fffffff;
-                const uint8_t* colbase = tiles + size_t(stage) * kOpBytes + half * kOpHalfBytes + sub;
+                const uint8_t* colbase = tiles + size_t(stage) * kOpBytes + half * kOpHalfBytes + row0 * 128 + sub;
                 float* dst = a.vsum + size_t(slab) * a.max_sent * kHeadDim + ch0;
                 int r = 0;
                 while (r < nrows) {
@@ -867,9 +869,9 @@ extern "C" int skipkv_score(const skipkv_shape* shape, const skipkv_params* para
     a1.so_smem = 0;
     a1.stages = int((max_smem - fixed1) / kOpBytes);
     if (a1.stages > kSwMaxStages) a1.stages = kSwMaxStages;
-    // sweep 2 also stages the current slab's sentence offsets and one sentence index per tile of the slab, when
+    // sweep 2 also stages the current slab's sentence offsets and one sentence index per 32 rows of the slab, when
     // that leaves at least two tile stages (otherwise its pooling warps read the table from global memory)
-    const size_t tab_bytes = (size_t(shape->max_sent) + 1 + size_t((shape->max_cap + 127) / 128)) * 4;
+    const size_t tab_bytes = (size_t(shape->max_sent) + 1 + size_t((shape->max_cap + 31) / 32)) * 4;
     a2.so_smem = (fixed1 + tab_bytes + 2 * kOpBytes <= max_smem) ? 1 : 0;
     const size_t fixed2 = fixed1 + (a2.so_smem ? tab_bytes : 0);
     a2.stages = int((max_smem - fixed2) / kOpBytes);
