@@ -59,6 +59,8 @@ compact_plan_kernel(int Hk, int max_sent, const int64_t* slab_off, const int32_t
                     int32_t* cp_run_dst) {
     __shared__ int wsum[kPlanThreads / 32][3];
     __shared__ int s_bad;
+    // the move kernel is launched as a programmatic dependent: let its CTAs set themselves up while this grid runs
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int slab = blockIdx.x;
     const int b = slab / Hk;
     const int tid = threadIdx.x;
@@ -141,13 +143,15 @@ compact_move_kernel(int n_slabs, int Hk, int max_sent, const int64_t* slab_off, 
     __shared__ uint32_t s_ticket;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
+    if (tid == 0) { mbar_init(&bar, 1); mbar_fence_init(); }
+    // everything below reads what the plan kernel wrote: wait until that grid has completed and its writes are visible
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     // every CTA derives the scheduler bound: the largest segment count of any slab
     int mx = 0;
     for (int i = tid; i < n_slabs; i += kMoveThreads) mx = max(mx, cp_nseg[i]);
 #pragma unroll
     for (int d = 16; d; d >>= 1) mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, d));
     if (lane == 0) s_red[warp] = mx;
-    if (tid == 0) { mbar_init(&bar, 1); mbar_fence_init(); }
     __syncthreads();
     int max_nseg = 0;
     for (int w = 0; w < kMoveThreads / 32; ++w) max_nseg = max(max_nseg, s_red[w]);
@@ -278,10 +282,22 @@ extern "C" int skipkv_compact(const skipkv_shape* shape, void* K, void* V, const
         SKIPKV_CUDA(cudaFuncSetAttribute(compact_move_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSegBytes));
         attr_set = true;
     }
-    const int grid = num_sms() * 3;
-    compact_move_kernel<<<grid, kMoveThreads, kSegBytes, st>>>(
-        L.slabs, shape->n_kv_heads, shape->max_sent, shape->slab_off, shape->cap, static_cast<__nv_bfloat16*>(K),
-        static_cast<__nv_bfloat16*>(V), index_map, hdr, nseg, loaded, nruns, run_src, run_dst);
-    SKIPKV_CUDA(cudaGetLastError());
+    // programmatic dependent launch: the move kernel's CTAs may start (and initialise) before the plan kernel has
+    // finished; they wait inside the kernel before touching the plan
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(unsigned(num_sms() * 3));
+    cfg.blockDim = dim3(kMoveThreads);
+    cfg.dynamicSmemBytes = kSegBytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr{};
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    SKIPKV_CUDA(cudaLaunchKernelEx(&cfg, compact_move_kernel, int(L.slabs), int(shape->n_kv_heads), int(shape->max_sent),
+                                   shape->slab_off, shape->cap, static_cast<__nv_bfloat16*>(K),
+                                   static_cast<__nv_bfloat16*>(V), index_map, hdr, static_cast<const int32_t*>(nseg), loaded,
+                                   static_cast<const int32_t*>(nruns), static_cast<const int32_t*>(run_src),
+                                   static_cast<const int32_t*>(run_dst)));
     return SKIPKV_OK;
 }
