@@ -95,6 +95,29 @@ int num_sms();
 // ---------------------------------------------------------------------------------------
 #ifdef __CUDACC__
 
+// Programmatic dependent launch between the kernels of one call: a kernel lets its successor's CTAs start early
+// (pdl_trigger, a no-op without a dependent), and the successor waits (pdl_wait, a no-op when launched normally)
+// until the predecessor grid has completed and its writes are visible, before it touches anything that grid wrote.
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+// host: launch `kernel` on `st` as a programmatic dependent of the kernel enqueued before it
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                    Args... args) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr{};
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 __device__ __forceinline__ size_t slab_row0(const int64_t* slab_off, const int32_t* cap, int Hk, int b, int h) {
     return size_t(slab_off[b]) * Hk + size_t(h) * cap[b];
 }

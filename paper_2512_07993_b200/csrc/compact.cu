@@ -60,7 +60,7 @@ compact_plan_kernel(int Hk, int max_sent, const int64_t* slab_off, const int32_t
     __shared__ int wsum[kPlanThreads / 32][3];
     __shared__ int s_bad;
     // the move kernel is launched as a programmatic dependent: let its CTAs set themselves up while this grid runs
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    pdl_trigger();
     const int slab = blockIdx.x;
     const int b = slab / Hk;
     const int tid = threadIdx.x;
@@ -145,7 +145,7 @@ compact_move_kernel(int n_slabs, int Hk, int max_sent, const int64_t* slab_off, 
 
     if (tid == 0) { mbar_init(&bar, 1); mbar_fence_init(); }
     // everything below reads what the plan kernel wrote: wait until that grid has completed and its writes are visible
-    asm volatile("griddepcontrol.wait;" ::: "memory");
+    pdl_wait();
     // every CTA derives the scheduler bound: the largest segment count of any slab
     int mx = 0;
     for (int i = tid; i < n_slabs; i += kMoveThreads) mx = max(mx, cp_nseg[i]);
@@ -284,20 +284,9 @@ extern "C" int skipkv_compact(const skipkv_shape* shape, void* K, void* V, const
     }
     // programmatic dependent launch: the move kernel's CTAs may start (and initialise) before the plan kernel has
     // finished; they wait inside the kernel before touching the plan
-    cudaLaunchConfig_t cfg{};
-    cfg.gridDim = dim3(unsigned(num_sms() * 3));
-    cfg.blockDim = dim3(kMoveThreads);
-    cfg.dynamicSmemBytes = kSegBytes;
-    cfg.stream = st;
-    cudaLaunchAttribute attr{};
-    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr.val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = &attr;
-    cfg.numAttrs = 1;
-    SKIPKV_CUDA(cudaLaunchKernelEx(&cfg, compact_move_kernel, int(L.slabs), int(shape->n_kv_heads), int(shape->max_sent),
-                                   shape->slab_off, shape->cap, static_cast<__nv_bfloat16*>(K),
-                                   static_cast<__nv_bfloat16*>(V), index_map, hdr, static_cast<const int32_t*>(nseg), loaded,
-                                   static_cast<const int32_t*>(nruns), static_cast<const int32_t*>(run_src),
-                                   static_cast<const int32_t*>(run_dst)));
+    SKIPKV_CUDA(launch_dependent(compact_move_kernel, dim3(unsigned(num_sms() * 3)), dim3(kMoveThreads), kSegBytes, st,
+                                 int(L.slabs), int(shape->n_kv_heads), int(shape->max_sent), shape->slab_off, shape->cap,
+                                 static_cast<__nv_bfloat16*>(K), static_cast<__nv_bfloat16*>(V), index_map, hdr, nseg, loaded,
+                                 nruns, run_src, run_dst));
     return SKIPKV_OK;
 }

@@ -167,6 +167,7 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_consta
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int G = gridDim.x, cta = blockIdx.x;
     const int n_slabs = a.n_slabs, Hk = a.Hk, RB = a.RB;
+    pdl_trigger();
     auto live = [&](int s) { return min(max(a.kv_len[s], 0), a.cap[s / Hk]); };
 
     if (tid == 0) {
@@ -212,6 +213,8 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_consta
         if (tid == kThreads - 1) pref[n_slabs] = int(run);
         __syncthreads();
     }
+    // (sweep 2) everything so far read only the call's inputs; what follows uses what sweep 1 wrote
+    pdl_wait();
     const uint32_t tmem_base = ctl->tmem_base;
     const int Ttot = pref[n_slabs];
     const int per_cta = max(1, (Ttot + G - 1) / G);
@@ -540,6 +543,8 @@ __global__ void __launch_bounds__(256)
 score_pool_kernel(int Hk, int max_sent, int max_cap, const int32_t* cap, const int32_t* kv_len,
                   const int32_t* sent_off, const int32_t* n_sent, float eps, const float* tok_imp_ws,
                   const float* vsum, float* sent_imp, __nv_bfloat16* vbar_hi, __nv_bfloat16* vbar_lo) {
+    pdl_trigger();
+    pdl_wait();
     const int slab = blockIdx.y;
     const int lane = threadIdx.x & 31;
     const int i = blockIdx.x * 8 + (threadIdx.x >> 5);
@@ -619,6 +624,7 @@ score_gram_kernel(const __grid_constant__ CUtensorMap mapHi, const __grid_consta
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int G = gridDim.x, cta = blockIdx.x;
     auto sent_of = [&](int s) { return min(max(n_sent[s], 0), max_sent); };
+    pdl_trigger();
 
     if (tid == 0) {
         mbar_init(&ctl->afull, 1);
@@ -660,6 +666,7 @@ score_gram_kernel(const __grid_constant__ CUtensorMap mapHi, const __grid_consta
         if (tid == kGramThreads - 1) ipref[n_slabs] = int(run);
         __syncthreads();
     }
+    pdl_wait();                                          // the pooled keys / row sums of the previous kernel
     const uint32_t tmem_base = ctl->tmem_base;
     const int n_items = ipref[n_slabs];
 
@@ -818,8 +825,12 @@ static int launch_sweep(const CUtensorMap& mapK, const CUtensorMap& mapQ, const 
                         cudaStream_t st) {
     auto kern = score_sweep_kernel<kSweep, kN>;
     SKIPKV_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
-    kern<<<grid, kSweep == 1 ? kSw1Threads : kSw2Threads, smem, st>>>(mapK, mapQ, a);
-    SKIPKV_CUDA(cudaGetLastError());
+    if (kSweep == 1) {
+        kern<<<grid, kSw1Threads, smem, st>>>(mapK, mapQ, a);
+        SKIPKV_CUDA(cudaGetLastError());
+    } else {
+        SKIPKV_CUDA(launch_dependent(kern, dim3(grid), dim3(kSw2Threads), smem, st, mapK, mapQ, a));
+    }
     return SKIPKV_OK;
 }
 
@@ -896,9 +907,9 @@ extern "C" int skipkv_score(const skipkv_shape* shape, const skipkv_params* para
     if (rc) return rc;
     {
         dim3 pgrid((shape->max_sent + 7) / 8, L.slabs);
-        score_pool_kernel<<<pgrid, 256, 0, st>>>(Hk, shape->max_sent, shape->max_cap, shape->cap, kv_len, sent_off,
-                                                 n_sent, params->eps, sc_tok, vsum, sent_imp, vbar_hi, vbar_lo);
-        SKIPKV_CUDA(cudaGetLastError());
+        SKIPKV_CUDA(launch_dependent(score_pool_kernel, pgrid, dim3(256), 0, st, Hk, shape->max_sent, shape->max_cap,
+                                     shape->cap, kv_len, sent_off, n_sent, params->eps, sc_tok, vsum, sent_imp, vbar_hi,
+                                     vbar_lo));
     }
     {
         const size_t gsmem = gram_smem_bytes(L.slabs);
@@ -907,14 +918,12 @@ extern "C" int skipkv_score(const skipkv_shape* shape, const skipkv_params* para
         const int ggrid = int(max_items < (long long)grid ? max_items : (long long)grid);
         SKIPKV_CUDA(cudaFuncSetAttribute(score_gram_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(gsmem)));
         SKIPKV_CUDA(cudaFuncSetAttribute(score_gram_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(gsmem)));
-        score_gram_kernel<1><<<ggrid, kGramThreads, gsmem, st>>>(mapHi, mapLo, L.slabs, shape->max_sent, n_sent, params->sigma,
-                                                                 params->tau, sc_z, sent_imp, sent_red, sent_lam, sent_score,
-                                                                 status);
-        SKIPKV_CUDA(cudaGetLastError());
-        score_gram_kernel<2><<<ggrid, kGramThreads, gsmem, st>>>(mapHi, mapLo, L.slabs, shape->max_sent, n_sent, params->sigma,
-                                                                 params->tau, sc_z, sent_imp, sent_red, sent_lam, sent_score,
-                                                                 status);
-        SKIPKV_CUDA(cudaGetLastError());
+        SKIPKV_CUDA(launch_dependent(score_gram_kernel<1>, dim3(ggrid), dim3(kGramThreads), gsmem, st, mapHi, mapLo, L.slabs,
+                                     shape->max_sent, n_sent, params->sigma, params->tau, sc_z, sent_imp, sent_red, sent_lam,
+                                     sent_score, status));
+        SKIPKV_CUDA(launch_dependent(score_gram_kernel<2>, dim3(ggrid), dim3(kGramThreads), gsmem, st, mapHi, mapLo, L.slabs,
+                                     shape->max_sent, n_sent, params->sigma, params->tau, sc_z, sent_imp, sent_red, sent_lam,
+                                     sent_score, status));
     }
     return SKIPKV_OK;
 }
