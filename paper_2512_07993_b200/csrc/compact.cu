@@ -61,6 +61,7 @@ compact_plan_kernel(int Hk, int max_sent, const int64_t* slab_off, const int32_t
     __shared__ int s_bad;
     // the move kernel is launched as a programmatic dependent: let its CTAs set themselves up while this grid runs
     pdl_trigger();
+    pdl_wait();                                          // inputs may come from the kernel before
     const int slab = blockIdx.x;
     const int b = slab / Hk;
     const int tid = threadIdx.x;
@@ -272,10 +273,9 @@ extern "C" int skipkv_compact(const skipkv_shape* shape, void* K, void* V, const
     int32_t* run_dst = reinterpret_cast<int32_t*>(w + L.cp_run_dst);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
 
-    compact_plan_kernel<<<L.slabs, kPlanThreads, 0, st>>>(shape->n_kv_heads, shape->max_sent, shape->slab_off,
-                                                          shape->cap, keep, sent_off, sent_id, n_sent, kv_len, hdr,
-                                                          nseg, loaded, nruns, run_src, run_dst);
-    SKIPKV_CUDA(cudaGetLastError());
+    SKIPKV_CUDA(launch_dependent(compact_plan_kernel, dim3(L.slabs), dim3(kPlanThreads), 0, st, int(shape->n_kv_heads),
+                                 int(shape->max_sent), shape->slab_off, shape->cap, keep, sent_off, sent_id, n_sent, kv_len,
+                                 hdr, nseg, loaded, nruns, run_src, run_dst));
 
     static thread_local bool attr_set = false;
     if (!attr_set) {

@@ -167,6 +167,7 @@ decode_attn_kernel(int batch, int Hq, int Hk, int n_slabs, const int64_t* slab_o
     int* pref = reinterpret_cast<int*>(sm + 1);                              // [n_slabs + 1] tile prefix
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    pdl_trigger();
     DEC_TRACE(0);
     auto live = [&](int s) { return min(max(kv_len[s], 0), cap[s / Hk]); };   // live rows of slab s
     const int n = Hq / Hk;                     // heads per group
@@ -179,6 +180,7 @@ decode_attn_kernel(int batch, int Hq, int Hk, int n_slabs, const int64_t* slab_o
         sm->is_last = 0;
         mbar_fence_init();
     }
+    pdl_wait();                                          // inputs (and the workspace) may come from the kernel before
     // tile prefix over slabs (block scan; every thread owns a contiguous block of slabs)
     {
         const int per = (n_slabs + kDecThreads - 1) / kDecThreads;
@@ -468,13 +470,13 @@ extern "C" int skipkv_decode_attn(const skipkv_shape* shape, const void* q, cons
     }
     int grid = num_sms() * kCtasPerSm;
     if (grid > L.dec_max_ctas) grid = L.dec_max_ctas;
-    decode_attn_kernel<<<grid, kDecThreads, smem, static_cast<cudaStream_t>(stream)>>>(
-        shape->batch, shape->n_q_heads, shape->n_kv_heads, L.slabs, shape->slab_off, shape->cap,
+    SKIPKV_CUDA(launch_dependent(
+        decode_attn_kernel, dim3(grid), dim3(kDecThreads), smem, static_cast<cudaStream_t>(stream), int(shape->batch),
+        int(shape->n_q_heads), int(shape->n_kv_heads), int(L.slabs), shape->slab_off, shape->cap,
         static_cast<const __nv_bfloat16*>(q), static_cast<const uint8_t*>(K), static_cast<const uint8_t*>(V), kv_len,
         static_cast<__nv_bfloat16*>(out), &reinterpret_cast<Header*>(w + L.header)->status,
-        reinterpret_cast<uint32_t*>(w + L.dec_cnt), reinterpret_cast<float*>(w + L.dec_part), shape->d_model,
-        static_cast<__nv_bfloat16*>(hidden), static_cast<const __nv_bfloat16*>(steer_vec), alpha, flag);
-    SKIPKV_CUDA(cudaGetLastError());
+        reinterpret_cast<uint32_t*>(w + L.dec_cnt), reinterpret_cast<float*>(w + L.dec_part), int(shape->d_model),
+        static_cast<__nv_bfloat16*>(hidden), static_cast<const __nv_bfloat16*>(steer_vec), alpha, flag));
     return SKIPKV_OK;
 }
 

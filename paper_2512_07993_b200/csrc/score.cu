@@ -168,6 +168,7 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_consta
     const int G = gridDim.x, cta = blockIdx.x;
     const int n_slabs = a.n_slabs, Hk = a.Hk, RB = a.RB;
     pdl_trigger();
+    if (kSweep == 1) pdl_wait();                         // first kernel of the call: its inputs may come from the kernel before
     auto live = [&](int s) { return min(max(a.kv_len[s], 0), a.cap[s / Hk]); };
 
     if (tid == 0) {
@@ -825,12 +826,7 @@ static int launch_sweep(const CUtensorMap& mapK, const CUtensorMap& mapQ, const 
                         cudaStream_t st) {
     auto kern = score_sweep_kernel<kSweep, kN>;
     SKIPKV_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
-    if (kSweep == 1) {
-        kern<<<grid, kSw1Threads, smem, st>>>(mapK, mapQ, a);
-        SKIPKV_CUDA(cudaGetLastError());
-    } else {
-        SKIPKV_CUDA(launch_dependent(kern, dim3(grid), dim3(kSw2Threads), smem, st, mapK, mapQ, a));
-    }
+    SKIPKV_CUDA(launch_dependent(kern, dim3(grid), dim3(kSweep == 1 ? kSw1Threads : kSw2Threads), smem, st, mapK, mapQ, a));
     return SKIPKV_OK;
 }
 

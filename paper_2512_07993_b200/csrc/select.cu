@@ -51,6 +51,8 @@ select_kernel(int max_sent, int P, int budget, int protect_tail, const float* se
     uint64_t* keys = reinterpret_cast<uint64_t*>(sel_smem);             // [P]
     uint8_t* flags = reinterpret_cast<uint8_t*>(keys + P);             // [P] keep flag by sentence index
     __shared__ uint32_t wsum[kSelThreads / 32];
+    pdl_trigger();
+    pdl_wait();                                          // inputs may come from the kernel before
     const int slab = blockIdx.x, tid = threadIdx.x;
     const float* score = sent_score + size_t(slab) * max_sent;
     const int32_t* so = sent_off + size_t(slab) * (max_sent + 1);
@@ -168,9 +170,8 @@ extern "C" int skipkv_select(const skipkv_shape* shape, const skipkv_params* par
         attr_smem = smem;
     }
     const int slabs = shape->batch * shape->n_kv_heads;
-    select_kernel<<<slabs, kSelThreads, smem, static_cast<cudaStream_t>(stream)>>>(
-        shape->max_sent, P, params->budget, params->protect_tail, sent_score, sent_off, n_sent, keep, kept_idx, n_kept,
-        new_len, &static_cast<Header*>(ws)->status);
-    SKIPKV_CUDA(cudaGetLastError());
+    SKIPKV_CUDA(launch_dependent(select_kernel, dim3(slabs), dim3(kSelThreads), smem, static_cast<cudaStream_t>(stream),
+                                 shape->max_sent, P, params->budget, params->protect_tail, sent_score, sent_off, n_sent, keep,
+                                 kept_idx, n_kept, new_len, &static_cast<Header*>(ws)->status));
     return SKIPKV_OK;
 }
