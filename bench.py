@@ -98,6 +98,22 @@ class ClockSampler:
                 "window": "warm-up + timed region" if t0 < self.t_start + 1e-3 else "timed region"}
 
 
+def max_over_ranks(values, dist, device):
+    """Element-wise maximum of a list of floats over all ranks (the replicas are independent: the slowest one
+    defines the job's time); identity without a process group."""
+    if dist is None:
+        return list(values)
+    tt = torch.tensor(list(values), device=device, dtype=torch.float64)
+    dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+    return tt.tolist()
+
+
+def replica_value(per_replica_us, world):
+    """Whole-job value for `world` independent replicas that each process one layer per per_replica_us:
+    microseconds per layer of the job = slowest replica's time / layers processed concurrently."""
+    return per_replica_us / world
+
+
 def oracle_shape(L):
     cfg = L["cfg"]
     return dict(batch=cfg.batch, Hq=cfg.n_q_heads, Hk=cfg.n_kv_heads, d=cfg.head_dim, alpha=cfg.window,
@@ -264,12 +280,7 @@ def main():
     us_med = {leg: statistics.median(v) for leg, v in per.items()}
     evict_us = us["score"] + us["select"] + us["compact"]
     step_ms = (evict_us + us["decode_attn"]) * NL / 1e3
-    if dist:
-        tt = torch.tensor([evict_us, step_ms, us["decode_attn"]], device="cuda", dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        evict_us, step_ms, dec_us_max = tt.tolist()
-    else:
-        dec_us_max = us["decode_attn"]
+    evict_us, step_ms, dec_us_max = max_over_ranks([evict_us, step_ms, us["decode_attn"]], dist, "cuda")
 
     # algorithmic bytes per layer from the actual lengths (mean over the NL layers)
     kv0 = np.stack([Ll["kv_len"].astype(np.int64) for Ll in Ls])
@@ -290,7 +301,7 @@ def main():
                      "frac_of_nominal_8TBs": gbs / 8000.0, "traffic": traffic.get(leg)}
     dominant = max(("score", "compact", "decode_attn"), key=lambda k: us[k])
 
-    line = {"metric": METRIC, "value": evict_us / world, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+    line = {"metric": METRIC, "value": replica_value(evict_us, world), "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": step_ms, "higher_is_better": False, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16 storage, f32 arithmetic", "data": "synthetic",
             "config": {"workload": f"configs[{args.config - 1}]: {cfg.name}", "batch": cfg.batch,
@@ -334,11 +345,8 @@ def main():
                 e2e_t.append((a.elapsed_time(b_) * 1e3, a.elapsed_time(c) * 1e3))
         e2e_evict = statistics.mean(x[0] for x in e2e_t)
         e2e_all = statistics.mean(x[1] for x in e2e_t)
-        if dist:
-            tt = torch.tensor([e2e_evict, e2e_all], device="cuda", dtype=torch.float64)
-            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-            e2e_evict, e2e_all = tt.tolist()
-        line["e2e"] = {"value": e2e_evict / world, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+        e2e_evict, e2e_all = max_over_ranks([e2e_evict, e2e_all], dist, "cuda")
+        line["e2e"] = {"value": replica_value(e2e_evict, world), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                        "whole_step_us": e2e_all / world,
                        "note": "host->device copy of K, V, queries and tables from pinned memory, the four calls, "
                                "device->host read of the attention output, hidden state and tables"}
