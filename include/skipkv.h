@@ -64,7 +64,8 @@ typedef struct {
     int32_t n_q_heads;    /* Hq                                                               */
     int32_t n_kv_heads;   /* Hk; Hq % Hk == 0, group n = Hq/Hk <= 8                           */
     int32_t head_dim;     /* must be 128                                                      */
-    int32_t window;       /* observation window alpha (recent queries), n*alpha <= 512        */
+    int32_t window;       /* observation window alpha (recent queries), n*alpha <= 512 and
+                             alpha <= 4 * floor(128 / n) (at most four query blocks per group) */
     int32_t d_model;      /* hidden size of the steering add; multiple of 8                   */
     int32_t max_sent;     /* row stride of the sentence tables; every n_sent <= max_sent      */
     int32_t max_cap;      /* host-known upper bound of cap[b] (sizes grids and the workspace) */
@@ -114,6 +115,10 @@ const char* skipkv_last_cuda_error(void);
  * tok_imp: device fp32, one value per cache row with the row indexing of K, nullable
  * (then it lives in the workspace).  sent_imp, sent_red, sent_lam, sent_score: device fp32
  * [batch][Hk][max_sent]; entries at i >= n_sent are not written.
+ * shape->total_rows must be the exact number of rows of the K buffer (the tiled copies are bounded by
+ * it).  The per-sentence sums are accumulated with floating-point atomics, so the last bits of the
+ * scores may differ from run to run.  The kernels of one call, and the first kernel of a call after
+ * the kernel before it on the stream, are launched as programmatic dependents: stream order holds.
  */
 int skipkv_score(const skipkv_shape* shape, const skipkv_params* params, const void* K,
                  const void* q_win, const int32_t* kv_len, const int32_t* sent_off,
@@ -196,8 +201,8 @@ int skipkv_append(const skipkv_shape* shape, void* K, void* V, const void* k_new
  * SKIPKV_ERR_UNSUPPORTED is returned, nothing is enqueued, and skipkv_last_cuda_error() says
  * which limit was exceeded.
  *
- * The first call on a device looks up the array's device address and sets a kernel attribute
- * (with that device current); make that first call before any stream capture begins.  Every call
+ * The first call on a device looks up the array's device address (with that device current);
+ * make that first call before any stream capture begins.  Every call
  * on a device shares the one array: each call first clears the counters it needs at zero (on
  * `stream`), and two calls whose GPU work overlaps (different streams, or different threads
  * without ordering between them) race on it and give undefined results.  Calls that follow one

@@ -80,7 +80,9 @@ def _check(rc: int, where: str):
 
 def make_shape(batch, n_q_heads, n_kv_heads, head_dim, window, d_model, max_sent, max_cap,
                slab_off: Optional[torch.Tensor], cap: Optional[torch.Tensor], total_rows: Optional[int] = None) -> Shape:
-    if total_rows is None:                      # an upper bound is enough for calls that never tile K
+    # total_rows must be the exact row count of the K / V buffers for skipkv_score (it bounds the tiled copies);
+    # the default is an upper bound, enough for workspace sizing and for the calls that never tile K
+    if total_rows is None:
         total_rows = batch * n_kv_heads * max_cap
     s = Shape(batch, n_q_heads, n_kv_heads, head_dim, window, d_model, max_sent, max_cap, total_rows,
               slab_off.data_ptr() if slab_off is not None else None,

@@ -277,13 +277,8 @@ extern "C" int skipkv_compact(const skipkv_shape* shape, void* K, void* V, const
                                  int(shape->max_sent), shape->slab_off, shape->cap, keep, sent_off, sent_id, n_sent, kv_len,
                                  hdr, nseg, loaded, nruns, run_src, run_dst));
 
-    static thread_local bool attr_set = false;
-    if (!attr_set) {
-        SKIPKV_CUDA(cudaFuncSetAttribute(compact_move_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSegBytes));
-        attr_set = true;
-    }
-    // programmatic dependent launch: the move kernel's CTAs may start (and initialise) before the plan kernel has
-    // finished; they wait inside the kernel before touching the plan
+    // set on every call: the attribute belongs to the current device's context, which a cached flag would not track
+    SKIPKV_CUDA(cudaFuncSetAttribute(compact_move_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSegBytes));
     SKIPKV_CUDA(launch_dependent(compact_move_kernel, dim3(unsigned(num_sms() * 3)), dim3(kMoveThreads), kSegBytes, st,
                                  int(L.slabs), int(shape->n_kv_heads), int(shape->max_sent), shape->slab_off, shape->cap,
                                  static_cast<__nv_bfloat16*>(K), static_cast<__nv_bfloat16*>(V), index_map, hdr, nseg, loaded,

@@ -463,11 +463,8 @@ extern "C" int skipkv_decode_attn(const skipkv_shape* shape, const void* q, cons
     uint8_t* w = static_cast<uint8_t*>(ws);
     const size_t smem = size_t(kStages) * 2 * kTileBytes + size_t(kConsWarps) * 4 * kWpStride * 4 + sizeof(DecSmem) +
                         size_t(L.slabs + 1) * 4;
-    static thread_local size_t attr_smem = 0;
-    if (smem > attr_smem) {
-        SKIPKV_CUDA(cudaFuncSetAttribute(decode_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
-        attr_smem = smem;
-    }
+    // set on every call: the attribute belongs to the current device's context, which a cached value would not track
+    SKIPKV_CUDA(cudaFuncSetAttribute(decode_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
     int grid = num_sms() * kCtasPerSm;
     if (grid > L.dec_max_ctas) grid = L.dec_max_ctas;
     SKIPKV_CUDA(launch_dependent(
@@ -510,18 +507,13 @@ static unsigned char* g_static_addr[kMaxDevices];      // device address of the 
 static bool g_static_ready[kMaxDevices];
 static std::mutex g_static_mutex;
 
-// First call on a device: resolve the array's device address and raise the kernel's dynamic
-// shared-memory limit.  Later calls only read the cached pointer.
+// First call on a device: resolve the array's device address.  Later calls only read the cached pointer.
 static int static_setup(int dev, unsigned char** base) {
     std::lock_guard<std::mutex> lock(g_static_mutex);
     if (!g_static_ready[dev]) {
         void* p = nullptr;
         SKIPKV_CUDA(cudaGetSymbolAddress(&p, g_static_scratch));
         if (!p) return SKIPKV_ERR_CUDA;
-        // the device's opt-in maximum: never below what any other caller of the kernel asked for
-        int optin = 0;
-        SKIPKV_CUDA(cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
-        SKIPKV_CUDA(cudaFuncSetAttribute(decode_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, optin));
         g_static_addr[dev] = static_cast<unsigned char*>(p);
         g_static_ready[dev] = true;
     }
@@ -560,6 +552,7 @@ extern "C" int skipkv_decode_attn_static(const skipkv_shape* shape, const void* 
                         size_t(slabs + 1) * 4;
     unsigned char* base = nullptr;
     if (int rc = static_setup(dev, &base)) return rc;
+    SKIPKV_CUDA(cudaFuncSetAttribute(decode_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     // The array keeps whatever the previous call left: the status word and the arrival counters
     // must start at zero (the partial records are fully written before they are read).

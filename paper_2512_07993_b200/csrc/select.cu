@@ -164,11 +164,8 @@ extern "C" int skipkv_select(const skipkv_shape* shape, const skipkv_params* par
     while (P < shape->max_sent) P <<= 1;
     const size_t smem = size_t(P) * 9;
     if (smem > 200 * 1024) return SKIPKV_ERR_UNSUPPORTED;     // max_sent beyond ~22k sentences per slab
-    static thread_local size_t attr_smem = 0;
-    if (smem > 48 * 1024 && smem > attr_smem) {
+    if (smem > 48 * 1024)   // set on every call: the attribute belongs to the current device's context
         SKIPKV_CUDA(cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
-        attr_smem = smem;
-    }
     const int slabs = shape->batch * shape->n_kv_heads;
     SKIPKV_CUDA(launch_dependent(select_kernel, dim3(slabs), dim3(kSelThreads), smem, static_cast<cudaStream_t>(stream),
                                  shape->max_sent, P, params->budget, params->protect_tail, sent_score, sent_off, n_sent, keep,
