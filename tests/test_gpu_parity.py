@@ -99,6 +99,64 @@ def test_score_matches_oracle(B, case):
             assert_close(f"tok_imp[{b},{h}]", tok[sl][:n], ref["tok_imp"][sl][:n])
 
 
+def with_empty_sentences(L, where=(0, 5, 17, 17, -1)):
+    """A copy of layer L whose sentence tables also hold zero-length sentences (a repeated offset)."""
+    cfg = L["cfg"]
+    ms = L["max_sent"] + len(where)
+    out = dict(L)
+    so = np.zeros((cfg.batch, cfg.n_kv_heads, ms + 1), np.int32)
+    sid = np.full((cfg.batch, cfg.n_kv_heads, ms), -1, np.int32)
+    ns = np.zeros_like(L["n_sent"])
+    for b in range(cfg.batch):
+        for h in range(cfg.n_kv_heads):
+            S = int(L["n_sent"][b, h])
+            off = list(L["sent_off"][b, h, :S + 1])
+            ids = list(L["sent_id"][b, h, :S])
+            for k, w in enumerate(sorted(x if x >= 0 else S for x in where)):
+                pos = min(w + k, len(off) - 1)
+                off.insert(pos, off[pos])                    # sentence `pos` becomes empty
+                ids.insert(pos, 1000 + k)
+            S2 = len(ids)
+            so[b, h, :S2 + 1] = off
+            so[b, h, S2 + 1:] = off[-1]
+            sid[b, h, :S2] = ids
+            ns[b, h] = S2
+    out.update(sent_off=so, sent_id=sid, n_sent=ns, max_sent=ms)
+    return out
+
+
+def test_score_and_eviction_with_empty_sentences(B):
+    """Zero-length sentences in the table: they pool to a zero key and zero importance, never own a row,
+    and vanish in compaction."""
+    L = with_empty_sentences(W.make_layer(W.config(1, name="empties", ctx_lo=1500, ctx_hi=1500, seed=21)))
+    cfg = L["cfg"]
+    ref = oracle_scores(L)
+    D = B.DeviceLayer(L)
+    D.score(); D.select(); D.compact(); D.decode_attn(steer=False)
+    torch.cuda.synchronize()
+    assert D.status() == 0
+    m = live_mask(L)
+    imp, red, lam, sc = (x.cpu().numpy() for x in (D.sent_imp, D.sent_red, D.sent_lam, D.sent_score))
+    assert_close("sent_imp", imp[m], ref["imp"][m])
+    assert_close("sent_red", red[m], ref["red"][m])
+    assert_close("sent_lam", lam[m], ref["lam"][m])
+    assert_close("sent_score", sc[m], ref["score"][m], rtol=1e-3, atol=1e-6)
+    sel = oracle.select_batch(ref["score"], L["sent_off"], L["n_sent"], cfg.budget, cfg.window)
+    assert np.array_equal(D.keep.cpu().numpy(), sel["keep"])
+    cmp_ = oracle.compact_batch(oshape(L), W.bf16_bits(L["K"]), W.bf16_bits(L["V"]), sel["keep"], L["sent_off"],
+                                L["sent_id"], L["n_sent"], L["kv_len"])
+    assert np.array_equal(D.kv_len.cpu().numpy(), cmp_["kv_len"])
+    assert np.array_equal(D.n_sent.cpu().numpy(), cmp_["n_sent"])
+    Kg = W.bf16_bits(D.K.cpu())
+    for b in range(cfg.batch):
+        for h in range(cfg.n_kv_heads):
+            sl = W.slab_rows(L, b, h)
+            n = int(cmp_["kv_len"][b, h])
+            assert np.array_equal(Kg[sl][:n], cmp_["K"][sl][:n])
+            k = int(cmp_["n_sent"][b, h])
+            assert np.array_equal(D.sent_off.cpu().numpy()[b, h, :k + 1], cmp_["sent_off"][b, h, :k + 1])
+
+
 # ----------------------------------------------------------------------------- select
 def near_tie_slabs(L, score, sel, rel=1e-5):
     """Slabs whose oracle scores at ranks k*..k*+2 (the cut neighbourhood) are closer than rel."""
