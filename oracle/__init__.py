@@ -134,6 +134,46 @@ def steer(hidden_bits, v_bits, alpha, flag):
     return h
 
 
+# ------------------------------------------------------------------ generation-space lookup table
+def lookup_table(H_bits, gen_off, tau, eps=1e-6):
+    """O9  Lookup table T (Section 4.1, "Sentence Similarity Score" and the sentence-score
+    table of Eq. "sentence-score-input"): sentence embeddings are the mean of the LAST-LAYER
+    hidden-state rows of each generation-space sentence (normalised as in O2), G is their
+    pairwise similarity (Eq. "PSS"), and T[i] = max_{j>i} G_ij when that exceeds tau, else 0
+    (the earlier sentence of a redundant pair is flagged, the later one kept).
+
+    H_bits uint16 [N, d_model] (bf16 bits, one sequence); gen_off int32 [S+1] CSR ranges of the
+    closed sentences.  Returns (T float64 [S], G float64 [S, S]).
+    """
+    H_bits = _c(H_bits, np.uint16); gen_off = _c(gen_off, np.int32)
+    _, vbar = pool(H_bits, gen_off, np.zeros(H_bits.shape[0], np.float64), eps)
+    G, _, T = gram_terms(vbar, tau)
+    return T, G
+
+
+def map_table(T, sent_id):
+    """O10  Phi (Eq. "sentence-score-cache"): the penalty of a cache-space sentence is the table
+    entry of the generation-space sentence it came from; a sentence without an entry (index
+    outside the table) carries no penalty."""
+    T = np.asarray(T, np.float64)
+    out = np.zeros(len(sent_id), np.float64)
+    for i, g in enumerate(np.asarray(sent_id).tolist()):
+        if 0 <= g < len(T):
+            out[i] = T[g]
+    return out
+
+
+def score_with_table(K_bits, Q_bits, sent_off, sent_id, T, sigma, tau, eps=1e-6):
+    """O11  Eq. "I_final" with the sentence penalty read from the table through Phi instead of
+    being derived from the pooled keys: importance (O1, O2) and redundancy (O3) as before.
+    Returns (imp, red, lam, score fp32)."""
+    tok = token_importance(K_bits, Q_bits)
+    imp, vbar = pool(K_bits, sent_off, tok, eps)
+    _, red, _ = gram_terms(vbar, tau)
+    lam = map_table(T, sent_id)
+    return imp, red, lam, final_score(imp, red, lam, sigma)
+
+
 # ------------------------------------------------------------------ batch drivers
 def score_batch(shape, K_bits, qwin_bits, kv_len, sent_off, n_sent, sigma, tau, eps, want_tok_imp=False):
     """shape: dict(batch,Hq,Hk,d,alpha,max_sent,slab_off,cap).  Returns dict of arrays."""

@@ -427,6 +427,87 @@ def test_o8_bit_exact_rounding():
 
 
 # ------------------------------------------------------------------ batch drivers == per-slab functions
+# ------------------------------------------------------------------ O9-O11 lookup table and Phi
+def test_o9_table_closed_form():
+    """Hand-built hidden states whose sentence means are known vectors."""
+    d = 8
+    e = np.eye(d)
+    c = 0.96
+    u = 24 * e[0] + 7 * e[1]                              # |u| = 25, cos(u, e0) = 0.96, exact in bf16
+    rows = [2 * e[0], 4 * e[0],                           # sentence 0: mean 3 e0
+            e[2], e[2], e[2],                             # sentence 1: e2
+            u + 0.5 * e[3], u - 0.5 * e[3],               # sentence 2: mean u (the e3 parts cancel)
+            8 * e[0]]                                     # sentence 3: e0 direction again
+    off = np.array([0, 2, 5, 7, 8], np.int32)
+    T, G = oracle.lookup_table(bits(np.array(rows)), off, 0.95, eps=0.0)
+    assert np.allclose(G[0], [1, 0, c, 1], atol=1e-15) and np.allclose(G[2, 3], c, atol=1e-15)
+    # sentence 0 repeats as sentence 3 (cos 1) and nearly as sentence 2 (0.96): the largest later one counts;
+    # sentence 2 is flagged through sentence 3; sentence 1 is unrelated; the last sentence has no later one
+    assert np.allclose(T, [1.0, 0.0, c, 0.0], atol=1e-15)
+    # with the threshold above 0.96 only the exact repeat is flagged
+    T2, _ = oracle.lookup_table(bits(np.array(rows)), off, 0.97, eps=0.0)
+    assert np.allclose(T2, [1.0, 0.0, 0.0, 0.0], atol=1e-15)
+    # mean pooling, not sum or last row: sentence 2 would otherwise not be the direction of u
+    assert np.allclose(G[2, 2], 1.0, atol=1e-15) and abs(G[1, 2]) < 1e-15
+
+
+def test_o9_matches_torch_and_incremental_form():
+    """Against torch fp64 ops, and against the running form (each closing sentence compared with
+    the earlier ones only, keeping the running maximum), which must give the same table."""
+    d, lens = 64, [3, 1, 7, 2, 5, 4, 1, 6]
+    off = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    H = rng.standard_normal((off[-1], d))
+    H[off[4]:off[5]] = H[off[0]:off[0] + 1] + 0.05 * rng.standard_normal((lens[4], d))  # 4 ~ first row of 0
+    H[off[6]:off[7]] = np.mean(H[off[2]:off[3]], axis=0)                                # 6 repeats 2's mean
+    Hb = bits(H)
+    tau = 0.5
+    T, G = oracle.lookup_table(Hb, off, tau)
+    Hd = torch.from_numpy(unbits(Hb))
+    m = torch.stack([Hd[off[i]:off[i + 1]].mean(dim=0) for i in range(len(lens))])
+    v = m / (m.norm(dim=1, keepdim=True) + 1e-6)
+    Gt = (v @ v.T).numpy()
+    assert np.allclose(G, Gt, atol=1e-13)
+    run = np.zeros(len(lens))
+    for j in range(len(lens)):
+        for i in range(j):
+            if Gt[i, j] > tau:
+                run[i] = max(run[i], Gt[i, j])
+    assert np.allclose(T, run, atol=1e-13)
+    assert T[2] > 0.99 and T[-1] == 0.0
+
+
+def test_o10_phi_lookup_and_compaction():
+    T = np.array([0.0, 0.97, 0.0, 0.99, 0.96])
+    assert np.array_equal(oracle.map_table(T, [3, 0, 4, 4, 1]), [0.99, 0.0, 0.96, 0.96, 0.97])
+    assert np.array_equal(oracle.map_table(T, [-1, 5, 2, 100]), [0, 0, 0, 0])     # no entry -> no penalty
+    # after an eviction the surviving cache-space sentences still find their own entries
+    d, lens = 8, [2, 3, 1, 4, 2]
+    off = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    K = bits(rng.standard_normal((off[-1], d))); V = bits(rng.standard_normal((off[-1], d)))
+    keep = np.array([1, 0, 1, 0, 1], np.uint8)
+    sid = np.arange(5, dtype=np.int32)
+    _, _, _, _, nsid = oracle.compact(K, V, keep, off, sid)
+    assert np.array_equal(oracle.map_table(T, nsid), oracle.map_table(T, sid)[keep == 1])
+
+
+def test_o11_score_with_table():
+    d, lens = 16, [4, 6, 3, 5]
+    off = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    K = bits(rng.standard_normal((off[-1], d))); Q = bits(rng.standard_normal((2, 3, d)))
+    T = np.array([0.0, 0.0, 0.98, 0.0, 0.0, 0.96])
+    sid = np.array([1, 2, 4, 5], np.int32)
+    imp, red, lam, sc = oracle.score_with_table(K, Q, off, sid, T, 0.1, 0.95)
+    tok = oracle.token_importance(K, Q)
+    imp0, vbar = oracle.pool(K, off, tok)
+    _, red0, lam_keys = oracle.gram_terms(vbar, 0.95)
+    assert np.array_equal(imp, imp0) and np.array_equal(red, red0)       # importance and redundancy unchanged
+    assert np.array_equal(lam, [0.0, 0.98, 0.0, 0.96]) and not lam_keys.any()
+    expect = (0.1 * imp - 0.9 * red - lam).astype(np.float32)
+    assert np.array_equal(sc, expect)
+    # a flagged sentence ranks below every unflagged one whatever its importance
+    assert sc[[1, 3]].max() < sc[[0, 2]].min()
+
+
 def test_batch_drivers_match_slab_functions():
     cfg = W.config(0)
     L = W.make_layer(cfg)
