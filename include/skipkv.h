@@ -10,6 +10,8 @@
  *   skipkv_compact      in-place packing of the surviving K/V rows + range-table update
  *   skipkv_decode_attn  GQA decode attention over the ragged, compacted cache
  *   skipkv_steer        steering-vector add on the hidden state
+ * and, beside them, the generation-space lookup table of the sentence penalty (skipkv_table_step)
+ * with the score variant that reads it (skipkv_score_table).
  *
  * Conventions
  *   - Every pointer marked "device" is a CUDA device pointer; "host" is ordinary memory.
@@ -183,6 +185,47 @@ int skipkv_steer(int32_t batch, int32_t d_model, void* hidden, const void* steer
  */
 int skipkv_append(const skipkv_shape* shape, void* K, void* V, const void* k_new, const void* v_new,
                   int32_t* kv_len, void* ws, void* stream);
+
+/*
+ * skipkv_table_step -- Section 4.1 "Sentence Similarity Score" and the lookup table T of Eq.
+ * "sentence-score-input", maintained one decode step at a time.  A sentence embedding is the mean of
+ * the LAST-LAYER hidden-state rows of the sentence's tokens (delimiter included), divided by
+ * (its 2-norm + eps); the similarity of two sentences is the dot product of their embeddings (Eq. "PSS");
+ * T[i] = max over later sentences j of that similarity when it exceeds tau, else 0 (the earlier sentence
+ * of a redundant pair is flagged, the later one kept).  Per sequence b this call
+ *   - adds hidden_last[b] to the running sum of the open sentence (acc, acc_count);
+ *   - if flag[b] != 0 (the token is a delimiter) closes the sentence: stores its embedding at
+ *     emb[b][n_gen_sent[b]], sets T[b][that index] = 0, increments n_gen_sent[b], clears the running sum,
+ *     writes the index to closed[b], and raises T[b][i] to the similarity with every earlier sentence i
+ *     whose similarity exceeds tau and the current entry;
+ *   - otherwise writes closed[b] = -1.
+ * After any number of steps T equals the one-shot definition over the closed sentences.
+ * hidden_last: device bf16 [batch][d_model] (read only).  flag: device u8 [batch].
+ * State, caller-owned, zero before the first step: acc device fp32 [batch][d_model], acc_count device int32
+ * [batch], n_gen_sent device int32 [batch].  emb: device fp32 [batch][max_gen_sent][d_model].
+ * lam_table: device fp32 [batch][max_gen_sent] (entries at and beyond n_gen_sent are not meaningful).
+ * closed: device int32 [batch] (output).  status: device uint32, nullable: SKIPKV_STATUS_BAD_TABLE is OR-ed
+ * in when a sentence closes with n_gen_sent == max_gen_sent (that sentence is dropped).
+ * d_model: multiple of 8, at most 16384; hidden_last, acc and emb 16-byte aligned.
+ */
+int skipkv_table_step(int32_t batch, int32_t d_model, int32_t max_gen_sent, const void* hidden_last,
+                      const uint8_t* flag, float* acc, int32_t* acc_count, float* emb, int32_t* n_gen_sent,
+                      int32_t* closed, float* lam_table, float tau, float eps, uint32_t* status, void* stream);
+
+/*
+ * skipkv_score_table -- skipkv_score with the sentence penalty taken from the lookup table through the
+ * mapping Phi of Eq. "sentence-score-cache" instead of the pooled keys:
+ *   sent_lam[i] = lam_table[b][sent_id[b][h][i]] if 0 <= sent_id[b][h][i] < table_len, else 0.
+ * Importance, redundancy and the final score are those of skipkv_score.  sent_id: device table (read
+ * only).  lam_table: device fp32 [batch][table_len] (row stride table_len), e.g. the table kept by
+ * skipkv_table_step with table_len = max_gen_sent.  Other arguments, limits and launch behaviour as
+ * skipkv_score.
+ */
+int skipkv_score_table(const skipkv_shape* shape, const skipkv_params* params, const void* K,
+                       const void* q_win, const int32_t* kv_len, const int32_t* sent_off,
+                       const int32_t* sent_id, const int32_t* n_sent, const float* lam_table,
+                       int32_t table_len, float* tok_imp, float* sent_imp, float* sent_red, float* sent_lam,
+                       float* sent_score, void* ws, void* stream);
 
 /*
  * skipkv_decode_attn_static -- skipkv_decode_attn for callers that cannot allocate device

@@ -21,7 +21,7 @@ ERRORS = {-1: "SKIPKV_ERR_INVALID_ARG", -2: "SKIPKV_ERR_UNSUPPORTED", -3: "SKIPK
           -4: "SKIPKV_ERR_CUDA", -5: "SKIPKV_ERR_TIMEOUT"}
 SYMBOLS = ["skipkv_workspace_bytes", "skipkv_workspace_init", "skipkv_status", "skipkv_last_cuda_error",
            "skipkv_score", "skipkv_select", "skipkv_compact", "skipkv_decode_attn", "skipkv_steer",
-           "skipkv_append", "skipkv_decode_attn_static"]
+           "skipkv_append", "skipkv_decode_attn_static", "skipkv_table_step", "skipkv_score_table"]
 
 
 class SkipKVError(RuntimeError):
@@ -155,6 +155,28 @@ def skipkv_append(shape, K, V, k_new, v_new, kv_len, ws, stream=None) -> None:
     _check(lib().skipkv_append(C.byref(shape), _ptr(K, torch.bfloat16), _ptr(V, torch.bfloat16),
                                _ptr(k_new, torch.bfloat16), _ptr(v_new, torch.bfloat16), _ptr(kv_len, torch.int32),
                                _ptr(ws), _stream(stream)), "skipkv_append")
+
+
+def skipkv_table_step(batch, d_model, max_gen_sent, hidden_last, flag, acc, acc_count, emb, n_gen_sent, closed,
+                      lam_table, tau, eps, status=None, stream=None) -> None:
+    _check(lib().skipkv_table_step(C.c_int32(batch), C.c_int32(d_model), C.c_int32(max_gen_sent),
+                                   _ptr(hidden_last, torch.bfloat16), _ptr(flag, torch.uint8),
+                                   _ptr(acc, torch.float32), _ptr(acc_count, torch.int32), _ptr(emb, torch.float32),
+                                   _ptr(n_gen_sent, torch.int32), _ptr(closed, torch.int32),
+                                   _ptr(lam_table, torch.float32), C.c_float(tau), C.c_float(eps),
+                                   _ptr(status, torch.int32), _stream(stream)), "skipkv_table_step")
+
+
+def skipkv_score_table(shape, params, K, q_win, kv_len, sent_off, sent_id, n_sent, lam_table, table_len, tok_imp,
+                       sent_imp, sent_red, sent_lam, sent_score, ws, stream=None) -> None:
+    _check(lib().skipkv_score_table(C.byref(shape), C.byref(params), _ptr(K, torch.bfloat16),
+                                    _ptr(q_win, torch.bfloat16), _ptr(kv_len, torch.int32),
+                                    _ptr(sent_off, torch.int32), _ptr(sent_id, torch.int32),
+                                    _ptr(n_sent, torch.int32), _ptr(lam_table, torch.float32),
+                                    C.c_int32(table_len), _ptr(tok_imp, torch.float32),
+                                    _ptr(sent_imp, torch.float32), _ptr(sent_red, torch.float32),
+                                    _ptr(sent_lam, torch.float32), _ptr(sent_score, torch.float32), _ptr(ws),
+                                    _stream(stream)), "skipkv_score_table")
 
 
 def skipkv_decode_attn_static(shape, q, K, V, kv_len, out, hidden, steer_vec, alpha, flag, status=None,

@@ -597,6 +597,16 @@ struct GramCtl {
 constexpr int kGramThreads = 6 * 32;
 static size_t gram_smem_bytes(int slabs) { return 1024 + 6 * size_t(kOpBytes) + sizeof(GramCtl) + size_t(slabs + 1) * 4; }
 
+// Optional source of the sentence penalty: the lookup table T of one value per generation-space sentence,
+// [batch][table_len], read through the cache-space sentence's generation-space index (Phi).  table == nullptr:
+// the penalty comes from the pooled keys of the slab.
+struct LamTable {
+    const float* table;
+    const int32_t* sent_id;
+    int table_len;
+    int Hk;
+};
+
 __device__ __forceinline__ bool gram_wait(GramCtl* ctl, uint64_t* bar, uint32_t parity, uint32_t* status) {
     if (mbar_try_wait(bar, parity)) return true;
     for (uint32_t i = 0; i < (1u << 22); ++i) {
@@ -615,7 +625,7 @@ template <int kPass>
 __global__ void __launch_bounds__(kGramThreads, 1)
 score_gram_kernel(const __grid_constant__ CUtensorMap mapHi, const __grid_constant__ CUtensorMap mapLo, int n_slabs,
                   int max_sent, const int32_t* n_sent, float sigma, float tau, float* sc_z, const float* sent_imp,
-                  float* sent_red, float* sent_lam, float* sent_score, uint32_t* status) {
+                  float* sent_red, float* sent_lam, float* sent_score, LamTable ext, uint32_t* status) {
     extern __shared__ uint8_t gram_smem_raw[];
     const uint32_t raw = smem_u32(gram_smem_raw);
     uint8_t* At = gram_smem_raw + (((raw + 1023u) & ~1023u) - raw);              // hi, lo of the i block
@@ -804,7 +814,12 @@ score_gram_kernel(const __grid_constant__ CUtensorMap mapHi, const __grid_consta
                 const size_t o = size_t(rowbase) + i;
                 if (kPass == 1) {
                     sc_z[o] = accum;
-                    sent_lam[o] = (mx > tau) ? mx : 0.f;
+                    if (ext.table) {                             // penalty from the generation-space table through Phi
+                        const int g = ext.sent_id[o];
+                        sent_lam[o] = (g >= 0 && g < ext.table_len) ? ext.table[size_t(slab / ext.Hk) * ext.table_len + g] : 0.f;
+                    } else {
+                        sent_lam[o] = (mx > tau) ? mx : 0.f;
+                    }
                 } else {
                     const float red = accum / float(S);
                     sent_red[o] = red;
@@ -834,10 +849,10 @@ static int launch_sweep(const CUtensorMap& mapK, const CUtensorMap& mapQ, const 
 
 using namespace skipkv;
 
-extern "C" int skipkv_score(const skipkv_shape* shape, const skipkv_params* params, const void* K, const void* q_win,
-                            const int32_t* kv_len, const int32_t* sent_off, const int32_t* n_sent, float* tok_imp,
-                            float* sent_imp, float* sent_red, float* sent_lam, float* sent_score, void* ws,
-                            void* stream) {
+static int score_impl(const skipkv_shape* shape, const skipkv_params* params, const void* K, const void* q_win,
+                      const int32_t* kv_len, const int32_t* sent_off, const int32_t* n_sent, float* tok_imp,
+                      float* sent_imp, float* sent_red, float* sent_lam, float* sent_score, LamTable ext, void* ws,
+                      void* stream) {
     if (int rc = check_shape(shape)) return rc;
     if (!params || !K || !q_win || !kv_len || !sent_off || !n_sent || !sent_imp || !sent_red || !sent_lam || !sent_score)
         return SKIPKV_ERR_INVALID_ARG;
@@ -916,10 +931,29 @@ extern "C" int skipkv_score(const skipkv_shape* shape, const skipkv_params* para
         SKIPKV_CUDA(cudaFuncSetAttribute(score_gram_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(gsmem)));
         SKIPKV_CUDA(launch_dependent(score_gram_kernel<1>, dim3(ggrid), dim3(kGramThreads), gsmem, st, mapHi, mapLo, L.slabs,
                                      shape->max_sent, n_sent, params->sigma, params->tau, sc_z, sent_imp, sent_red, sent_lam,
-                                     sent_score, status));
+                                     sent_score, ext, status));
         SKIPKV_CUDA(launch_dependent(score_gram_kernel<2>, dim3(ggrid), dim3(kGramThreads), gsmem, st, mapHi, mapLo, L.slabs,
                                      shape->max_sent, n_sent, params->sigma, params->tau, sc_z, sent_imp, sent_red, sent_lam,
-                                     sent_score, status));
+                                     sent_score, ext, status));
     }
     return SKIPKV_OK;
+}
+
+extern "C" int skipkv_score(const skipkv_shape* shape, const skipkv_params* params, const void* K, const void* q_win,
+                            const int32_t* kv_len, const int32_t* sent_off, const int32_t* n_sent, float* tok_imp,
+                            float* sent_imp, float* sent_red, float* sent_lam, float* sent_score, void* ws,
+                            void* stream) {
+    return score_impl(shape, params, K, q_win, kv_len, sent_off, n_sent, tok_imp, sent_imp, sent_red, sent_lam,
+                      sent_score, LamTable{nullptr, nullptr, 0, 1}, ws, stream);
+}
+
+extern "C" int skipkv_score_table(const skipkv_shape* shape, const skipkv_params* params, const void* K,
+                                  const void* q_win, const int32_t* kv_len, const int32_t* sent_off,
+                                  const int32_t* sent_id, const int32_t* n_sent, const float* lam_table,
+                                  int32_t table_len, float* tok_imp, float* sent_imp, float* sent_red, float* sent_lam,
+                                  float* sent_score, void* ws, void* stream) {
+    if (!sent_id || !lam_table || table_len <= 0) return SKIPKV_ERR_INVALID_ARG;
+    if (int rc = check_shape(shape)) return rc;
+    return score_impl(shape, params, K, q_win, kv_len, sent_off, n_sent, tok_imp, sent_imp, sent_red, sent_lam,
+                      sent_score, LamTable{lam_table, sent_id, table_len, shape->n_kv_heads}, ws, stream);
 }

@@ -28,7 +28,7 @@ import numpy as np
 import torch
 
 # stream kinds (sub-keys of the Philox seed sequence)
-_K_STRUCT, _K_KEYS, _K_VALS, _K_NOISE, _K_QWIN, _K_QDEC, _K_HID, _K_STEER, _K_LENS, _K_MISC = range(10)
+_K_STRUCT, _K_KEYS, _K_VALS, _K_NOISE, _K_QWIN, _K_QDEC, _K_HID, _K_STEER, _K_LENS, _K_MISC, _K_GEN, _K_GENNOISE = range(12)
 
 
 @dataclass(frozen=True)
@@ -217,3 +217,34 @@ def slab_rows(layer: Dict[str, object], b: int, h: int) -> slice:
     cfg = layer["cfg"]
     r0 = int(layer["slab_off"][b]) * cfg.n_kv_heads + h * int(layer["cap"][b])
     return slice(r0, r0 + int(layer["cap"][b]))
+
+
+def make_generation(cfg: Workload, steps: int, d_model: Optional[int] = None, noise_hi: float = 0.6) -> Dict[str, object]:
+    """Last-layer hidden states of ``steps`` generated tokens per sequence, with sentence structure.
+
+    Sentences are drawn as for the cache (same length distribution and duplicate rate).  Tokens of a fresh
+    sentence are N(0,1); a duplicate sentence is its source plus N(0, s^2) noise with s uniform in
+    [0, noise_hi], so that the cosine of the two sentence means, about 1/sqrt(1+s^2), falls on both sides
+    of the usual threshold.  The last sentence of every even sequence is left open (no closing delimiter).
+    Returns H bf16 ``[batch, steps, d_model]``, flag uint8 ``[steps, batch]`` (1 = the token closes a
+    sentence) and gen_off (per sequence, int32 CSR ranges of the closed sentences).
+    """
+    dm = cfg.d_model if d_model is None else d_model
+    H = torch.zeros((cfg.batch, steps, dm), dtype=torch.bfloat16)
+    flag = np.zeros((steps, cfg.batch), np.uint8)
+    gen_off = []
+    for b in range(cfg.batch):
+        lengths, dup_src = draw_sentences(cfg, 0, b, steps)
+        off = np.concatenate([[0], np.cumsum(lengths)]).astype(np.int32)
+        h = to_bf16(_rng(cfg.seed, 0, b, _K_GEN).standard_normal((steps, dm), dtype=np.float32))
+        z = _rng(cfg.seed, 0, b, _K_GENNOISE)
+        for i in np.nonzero(dup_src >= 0)[0]:
+            s0, ln = int(dup_src[i]), int(lengths[i])
+            sd = float(z.uniform(0.0, noise_hi))
+            noise = torch.from_numpy(z.standard_normal((ln, dm), dtype=np.float32))
+            h[off[i]:off[i] + ln] = (h[off[s0]:off[s0] + ln].float() + sd * noise).to(torch.bfloat16)
+        H[b] = h
+        n_closed = len(lengths) - (1 if b % 2 == 0 else 0)
+        flag[off[1:n_closed + 1] - 1, b] = 1
+        gen_off.append(off[:n_closed + 1].copy())
+    return dict(H=H, flag=flag, gen_off=gen_off, d_model=dm, steps=steps)
