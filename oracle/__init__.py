@@ -174,6 +174,71 @@ def score_with_table(K_bits, Q_bits, sent_off, sent_id, T, sigma, tau, eps=1e-6)
     return imp, red, lam, final_score(imp, red, lam, sigma)
 
 
+# ------------------------------------------------------------------ exactly-B retention
+def select_fill(score, sent_off, tok_imp, budget, protect_tail):
+    """O12  Selection that retains exactly B tokens (Section 4.1: tokens are evicted in increasing
+    order of the final score until the cache meets the budget).  Whole sentences are kept in rank
+    order as in O5; the first sentence that does not fit (the cut sentence) then gives up only its
+    lowest-scoring tokens: redundancy and penalty are the same for all tokens of a sentence, so
+    inside it the final-score order is the token-importance order.  Its `slack = B - kept` tokens of
+    largest tok_imp survive (equal values: the earlier token first).
+
+    score fp32 [S], sent_off int32 [S+1], tok_imp fp32 [N].  Returns (keep uint8 [S] with 1 = whole
+    sentence kept, 2 = cut sentence partly kept; tok_keep uint8 [N]; new_len)."""
+    score = np.asarray(score, np.float32); sent_off = np.asarray(sent_off, np.int64)
+    tok_imp = np.asarray(tok_imp, np.float32)
+    S = len(sent_off) - 1
+    total = int(sent_off[S]) if S > 0 else 0
+    keep = np.zeros(S, np.uint8); tok_keep = np.zeros(total, np.uint8)
+    if total <= budget:
+        keep[:] = 1; tok_keep[:] = 1
+        return keep, tok_keep, total
+    forced = [protect_tail > 0 and sent_off[i + 1] > total - protect_tail and sent_off[i + 1] > sent_off[i]
+              for i in range(S)]
+    order = [i for i in range(S) if forced[i]]
+    order += sorted((i for i in range(S) if not forced[i]), key=lambda i: (-float(score[i]), i))
+    kept = 0
+    for i in order:
+        b, e = int(sent_off[i]), int(sent_off[i + 1])
+        if kept + (e - b) > budget:
+            slack = budget - kept
+            if slack > 0:
+                best = sorted(range(b, e), key=lambda t: (-float(tok_imp[t]), t))[:slack]
+                tok_keep[best] = 1
+                keep[i] = 2
+            break
+        kept += e - b
+        keep[i] = 1
+        tok_keep[b:e] = 1
+    return keep, tok_keep, int(tok_keep.sum())
+
+
+def compact_tokens(K_bits, V_bits, tok_keep, sent_off, sent_id):
+    """O13  Compaction with token-level survivors (Section 4.1, "Updating Cache Ranges After
+    Eviction", Eq. "after", evaluated literally): survivors p_1 < ... < p_B' are the kept token
+    indices; row k of the new cache is old row p_k; sentence (b, e) (inclusive ends) becomes
+    (min{k : p_k >= b}, max{k : p_k <= e}) and disappears when no survivor lies inside it.
+    Returns (K, V, index_map, new sent_off CSR, new sent_id)."""
+    K_bits = _c(K_bits, np.uint16); V_bits = _c(V_bits, np.uint16)
+    p = [t for t in range(len(tok_keep)) if tok_keep[t]]
+    new_off = [0]; new_id = []
+    for i in range(len(sent_off) - 1):
+        b, e = int(sent_off[i]), int(sent_off[i + 1]) - 1
+        if e < b:
+            continue
+        lo = [k for k, pk in enumerate(p) if pk >= b]
+        hi = [k for k, pk in enumerate(p) if pk <= e]
+        if not lo or not hi or min(lo) > max(hi):
+            continue
+        if min(lo) != new_off[-1]:
+            raise AssertionError("remapped ranges are not contiguous")
+        new_off.append(max(hi) + 1)
+        new_id.append(int(sent_id[i]))
+    idx = np.asarray(p, np.int64)
+    return (K_bits[idx], V_bits[idx], idx.astype(np.int32), np.asarray(new_off, np.int32),
+            np.asarray(new_id, np.int32))
+
+
 # ------------------------------------------------------------------ batch drivers
 def score_batch(shape, K_bits, qwin_bits, kv_len, sent_off, n_sent, sigma, tau, eps, want_tok_imp=False):
     """shape: dict(batch,Hq,Hk,d,alpha,max_sent,slab_off,cap).  Returns dict of arrays."""

@@ -508,6 +508,104 @@ def test_o11_score_with_table():
     assert sc[[1, 3]].max() < sc[[0, 2]].min()
 
 
+# ------------------------------------------------------------------ O12-O13 exactly-B retention
+def test_o12_hand_example():
+    lens = [3, 4, 2, 5]
+    off = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    score = np.array([0.5, 0.1, 0.9, 0.3], np.float32)          # rank: 2, 0, 3, 1
+    tok = np.zeros(14, np.float32)
+    tok[9:14] = [0.2, 0.7, 0.7, 0.1, 0.4]                        # sentence 3
+    # budget 8: sentences 2 and 0 fit (5 tokens); sentence 3 (5 tokens) does not: its 3 best tokens stay,
+    # the tie 0.7 / 0.7 keeps both, then 0.4
+    keep, tk, nl = oracle.select_fill(score, off, tok, 8, 0)
+    assert np.array_equal(keep, [1, 0, 1, 2]) and nl == 8
+    assert np.array_equal(np.nonzero(tk)[0], [0, 1, 2, 7, 8, 10, 11, 13])
+    # budget 7: two tokens of the cut sentence; among the equal pair the earlier comes first, both fit
+    keep, tk, nl = oracle.select_fill(score, off, tok, 7, 0)
+    assert np.array_equal(np.nonzero(tk)[0], [0, 1, 2, 7, 8, 10, 11]) and nl == 7
+    # budget 6: one token: the earlier of the equal pair
+    keep, tk, nl = oracle.select_fill(score, off, tok, 6, 0)
+    assert np.array_equal(np.nonzero(tk)[0], [0, 1, 2, 7, 8, 10]) and keep[3] == 2
+    # budget 5: no slack, nothing partial: identical to the whole-sentence rule
+    keep, tk, nl = oracle.select_fill(score, off, tok, 5, 0)
+    assert np.array_equal(keep, [1, 0, 1, 0]) and nl == 5
+    # fits already
+    keep, tk, nl = oracle.select_fill(score, off, tok, 14, 0)
+    assert keep.all() and tk.all() and nl == 14
+
+
+def test_o12_random_properties():
+    r = np.random.default_rng(7)
+    for trial in range(60):
+        S = int(r.integers(1, 12))
+        lens = r.integers(0, 7, size=S)
+        off = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+        N = int(off[-1])
+        score = r.choice(np.array([-1.0, -0.5, 0.0, 0.25, 0.5], np.float32), size=S)
+        tok = r.choice(np.array([0.0, 0.1, 0.2, 0.3], np.float32), size=N)
+        budget = int(r.integers(0, N + 2)); pt = int(r.integers(0, 4))
+        keep, tk, nl = oracle.select_fill(score, off, tok, budget, pt)
+        k5, _, nl5 = oracle.select(score, off, budget, pt)
+        assert np.array_equal(keep == 1, k5 == 1)                 # the whole sentences are those of O5
+        assert nl == int(tk.sum()) and nl5 <= nl <= max(budget, nl5)
+        if N > budget:
+            assert nl == budget                                   # exactly B
+        cut = np.nonzero(keep == 2)[0]
+        assert len(cut) <= 1
+        for i in range(S):
+            span = tk[off[i]:off[i + 1]]
+            if keep[i] == 1: assert span.all()
+            if keep[i] == 0: assert not span.any()
+        if len(cut):
+            c = int(cut[0]); b, e = int(off[c]), int(off[c + 1])
+            inside, outside = tok[b:e][tk[b:e] == 1], tok[b:e][tk[b:e] == 0]
+            assert 0 < len(inside) < e - b
+            assert inside.min() >= outside.max()                  # no evicted token outranks a kept one
+            # among equal values the earlier tokens are the kept ones
+            v = inside.min()
+            eq = np.nonzero(tok[b:e] == v)[0]
+            flags = tk[b:e][eq]
+            assert (np.diff(flags.astype(int)) <= 0).all()
+
+
+def test_o13_matches_o6_and_gather():
+    r = np.random.default_rng(11)
+    d = 8
+    for trial in range(30):
+        S = int(r.integers(1, 9))
+        lens = r.integers(0, 6, size=S)
+        off = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+        N = int(off[-1])
+        K = bits(r.standard_normal((max(N, 1), d)))[:N]; V = bits(r.standard_normal((max(N, 1), d)))[:N]
+        sid = r.permutation(50)[:S].astype(np.int32)
+        # whole-sentence survivors: must agree with the sentence-level compaction
+        keep = r.integers(0, 2, size=S).astype(np.uint8)
+        tk = np.zeros(N, np.uint8)
+        for i in range(S):
+            tk[off[i]:off[i + 1]] = keep[i]
+        Ko, Vo, im, nso, nsid = oracle.compact_tokens(K, V, tk, off, sid)
+        if N:
+            K6, V6, im6, nso6, nsid6 = oracle.compact(K, V, keep, off, sid)
+            assert np.array_equal(Ko, K6) and np.array_equal(Vo, V6) and np.array_equal(im, im6)
+            assert np.array_equal(nso, nso6) and np.array_equal(nsid, nsid6)
+        # arbitrary token survivors: numpy gather and per-sentence counts
+        tk = r.integers(0, 2, size=N).astype(np.uint8)
+        Ko, Vo, im, nso, nsid = oracle.compact_tokens(K, V, tk, off, sid)
+        assert np.array_equal(Ko, K[tk == 1]) and np.array_equal(Vo, V[tk == 1])
+        assert np.array_equal(im, np.nonzero(tk)[0])
+        counts = np.array([int(tk[off[i]:off[i + 1]].sum()) for i in range(S)])
+        assert np.array_equal(np.diff(nso), counts[counts > 0]) and np.array_equal(nsid, sid[counts > 0])
+
+
+def test_o13_hand_example():
+    off = np.array([0, 3, 5, 9], np.int32)
+    K = bits(np.arange(9 * 2).reshape(9, 2)); V = bits(-np.arange(9 * 2).reshape(9, 2))
+    tk = np.array([1, 1, 1, 0, 0, 0, 1, 0, 1], np.uint8)          # sentence 1 evicted, sentence 2 keeps tokens 6 and 8
+    Ko, Vo, im, nso, nsid = oracle.compact_tokens(K, V, tk, off, np.array([4, 5, 6], np.int32))
+    assert np.array_equal(im, [0, 1, 2, 6, 8]) and np.array_equal(nso, [0, 3, 5]) and np.array_equal(nsid, [4, 6])
+    assert np.array_equal(unbits(Ko)[:, 0], [0, 2, 4, 12, 16])
+
+
 def test_batch_drivers_match_slab_functions():
     cfg = W.config(0)
     L = W.make_layer(cfg)
