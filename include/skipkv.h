@@ -11,7 +11,8 @@
  *   skipkv_decode_attn  GQA decode attention over the ragged, compacted cache
  *   skipkv_steer        steering-vector add on the hidden state
  * and, beside them, the generation-space lookup table of the sentence penalty (skipkv_table_step)
- * with the score variant that reads it (skipkv_score_table).
+ * with the score variant that reads it (skipkv_score_table), and the variants of select and compact that
+ * retain exactly B tokens (skipkv_select_fill, skipkv_compact_fill).
  *
  * Conventions
  *   - Every pointer marked "device" is a CUDA device pointer; "host" is ordinary memory.
@@ -226,6 +227,32 @@ int skipkv_score_table(const skipkv_shape* shape, const skipkv_params* params, c
                        const int32_t* sent_id, const int32_t* n_sent, const float* lam_table,
                        int32_t table_len, float* tok_imp, float* sent_imp, float* sent_red, float* sent_lam,
                        float* sent_score, void* ws, void* stream);
+
+/*
+ * skipkv_select_fill, skipkv_compact_fill -- Section 4.1 taken to exactly B survivors (tokens leave in
+ * increasing order of the final score until the cache meets the budget).  skipkv_select_fill keeps whole
+ * sentences as skipkv_select does; the first sentence of the ranking that does not fit (the cut sentence)
+ * then keeps its slack = B - kept tokens of largest tok_imp -- redundancy and penalty are constant inside a
+ * sentence, so there the final-score order is the importance order; equal values: the earlier token.  That
+ * sentence gets keep = 2 and its tokens are flagged in tok_keep (device u8, one byte per cache row with the
+ * row indexing of K; only the bytes of a cut sentence are written or meaningful).  new_len is B for every
+ * slab that was over the budget (when slack is 0 nothing is cut and the result is that of skipkv_select).
+ * tok_imp: device fp32 per cache row as written by skipkv_score, or NULL to use the copy that the last
+ * skipkv_score call left in this workspace.  Other arguments as skipkv_select.
+ *
+ * skipkv_compact_fill is skipkv_compact for such a selection: a sentence with keep = 2 survives with its
+ * flagged tokens only, in order; ranges follow Eq. "after" (b <- min{k : p_k >= b}, e <- max{k : p_k <= e}
+ * over the survivor list p), so the cut sentence stays in the tables with its shortened length, and
+ * index_map names each survivor's old token index.  At most 4 sentences with keep = 2 per slab (more:
+ * SKIPKV_STATUS_BAD_TABLE and that slab is left unmoved).  tok_keep is read only.
+ */
+int skipkv_select_fill(const skipkv_shape* shape, const skipkv_params* params, const float* sent_score,
+                       const float* tok_imp, const int32_t* sent_off, const int32_t* n_sent, uint8_t* keep,
+                       uint8_t* tok_keep, int32_t* kept_idx, int32_t* n_kept, int32_t* new_len, void* ws,
+                       void* stream);
+int skipkv_compact_fill(const skipkv_shape* shape, void* K, void* V, const uint8_t* keep,
+                        const uint8_t* tok_keep, int32_t* sent_off, int32_t* sent_id, int32_t* n_sent,
+                        int32_t* kv_len, int32_t* index_map, void* ws, void* stream);
 
 /*
  * skipkv_decode_attn_static -- skipkv_decode_attn for callers that cannot allocate device

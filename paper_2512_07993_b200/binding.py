@@ -21,7 +21,8 @@ ERRORS = {-1: "SKIPKV_ERR_INVALID_ARG", -2: "SKIPKV_ERR_UNSUPPORTED", -3: "SKIPK
           -4: "SKIPKV_ERR_CUDA", -5: "SKIPKV_ERR_TIMEOUT"}
 SYMBOLS = ["skipkv_workspace_bytes", "skipkv_workspace_init", "skipkv_status", "skipkv_last_cuda_error",
            "skipkv_score", "skipkv_select", "skipkv_compact", "skipkv_decode_attn", "skipkv_steer",
-           "skipkv_append", "skipkv_decode_attn_static", "skipkv_table_step", "skipkv_score_table"]
+           "skipkv_append", "skipkv_decode_attn_static", "skipkv_table_step", "skipkv_score_table",
+           "skipkv_select_fill", "skipkv_compact_fill"]
 
 
 class SkipKVError(RuntimeError):
@@ -177,6 +178,24 @@ def skipkv_score_table(shape, params, K, q_win, kv_len, sent_off, sent_id, n_sen
                                     _ptr(sent_imp, torch.float32), _ptr(sent_red, torch.float32),
                                     _ptr(sent_lam, torch.float32), _ptr(sent_score, torch.float32), _ptr(ws),
                                     _stream(stream)), "skipkv_score_table")
+
+
+def skipkv_select_fill(shape, params, sent_score, tok_imp, sent_off, n_sent, keep, tok_keep, kept_idx, n_kept, new_len,
+                       ws, stream=None) -> None:
+    _check(lib().skipkv_select_fill(C.byref(shape), C.byref(params), _ptr(sent_score, torch.float32),
+                                    _ptr(tok_imp, torch.float32), _ptr(sent_off, torch.int32),
+                                    _ptr(n_sent, torch.int32), _ptr(keep, torch.uint8), _ptr(tok_keep, torch.uint8),
+                                    _ptr(kept_idx, torch.int32), _ptr(n_kept, torch.int32),
+                                    _ptr(new_len, torch.int32), _ptr(ws), _stream(stream)), "skipkv_select_fill")
+
+
+def skipkv_compact_fill(shape, K, V, keep, tok_keep, sent_off, sent_id, n_sent, kv_len, index_map, ws,
+                        stream=None) -> None:
+    _check(lib().skipkv_compact_fill(C.byref(shape), _ptr(K, torch.bfloat16), _ptr(V, torch.bfloat16),
+                                     _ptr(keep, torch.uint8), _ptr(tok_keep, torch.uint8),
+                                     _ptr(sent_off, torch.int32), _ptr(sent_id, torch.int32),
+                                     _ptr(n_sent, torch.int32), _ptr(kv_len, torch.int32),
+                                     _ptr(index_map, torch.int32), _ptr(ws), _stream(stream)), "skipkv_compact_fill")
 
 
 def skipkv_decode_attn_static(shape, q, K, V, kv_len, out, hidden, steer_vec, alpha, flag, status=None,

@@ -39,6 +39,7 @@ struct WsLayout {
     size_t sc_vbar_hi;     // bf16   [slabs][max_sent][128]  normalised mean key, high part
     size_t sc_vbar_lo;     // bf16   [slabs][max_sent][128]  and the rounding remainder
     size_t sc_z;           // float  [slabs][max_sent]
+    size_t cp_part;        // int32  [slabs][1 + 3*kMaxPartial]  partly kept sentences: count, then (begin, end, dst)
     size_t total;
     int slabs, group, qrows, dec_max_ctas;
     int sc_wb;             // window positions per query block: floor(128 / group)
@@ -47,6 +48,7 @@ struct WsLayout {
 
 constexpr int kDecMaxCtas = 1024;     // upper bound of the persistent grids
 constexpr int kMaxQueryBlocks = 4;
+constexpr int kMaxPartial = 4;        // partly kept sentences per slab that one compaction call can carry
 
 inline size_t align256(size_t x) { return (x + 255) & ~size_t(255); }
 
@@ -75,6 +77,7 @@ inline WsLayout make_layout(const skipkv_shape& s) {
     L.sc_vbar_hi = take(slabs * ms * kHeadDim * 2);
     L.sc_vbar_lo = take(slabs * ms * kHeadDim * 2);
     L.sc_z = take(slabs * ms * 4);
+    L.cp_part = take(slabs * (1 + 3 * kMaxPartial) * 4);
     L.total = o;
     return L;
 }

@@ -13,6 +13,11 @@
 //         register staging), publishes "segments 0..j of this stream are loaded", and then
 //         writes the pieces to their destination with bulk stores.
 //
+// With partly kept sentences (skipkv_compact_fill: keep == 2, survivors flagged per token) the plan first packs
+// the surviving rows of such a sentence to the front of the sentence's own rows, so that it becomes a shorter
+// contiguous sentence and the move proceeds unchanged; a third, tiny launch then corrects the index-map
+// entries of those sentences.
+//
 // Why this is safe in place: rows only move down (dst <= src), so a store into segment j can
 // only overwrite source rows of segments <= j.  A segment therefore stores only after every
 // lower segment of its stream has finished loading (the per-stream `loaded` counter advances
@@ -52,13 +57,43 @@ __device__ __forceinline__ void block_scan3(int v0, int v1, int v2, int& e0, int
     __syncthreads();
 }
 
+// Rows of tokens [pb, pe) of a slab whose flag is set move, in order, to rows pb, pb+1, ... of the same slab.
+// K and V together, 64 rows per pass: every thread holds one 16-byte piece of each; all pieces of a pass are read before any is written,
+// and destinations never lie above sources.
+__device__ __forceinline__ void pack_rows(uint4* kbase, uint4* vbase, const uint8_t* tk, int pb, int pe, int* s_pos,
+                                          int* s_wcnt) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int r = tid >> 4, col = tid & 15;
+    int done = 0;
+    for (int cb = pb; cb < pe; cb += 64) {
+        if (tid < 64) {
+            const int f = (cb + tid < pe) ? (tk[cb + tid] != 0) : 0;
+            const unsigned m = __ballot_sync(0xffffffffu, f);
+            s_pos[tid] = __popc(m & ((1u << lane) - 1u));
+            if (lane == 0) s_wcnt[warp] = __popc(m);
+        }
+        __syncthreads();
+        const int t = cb + r;
+        const bool f = t < pe && tk[t] != 0;
+        const int dst = pb + done + s_pos[r] + (r >= 32 ? s_wcnt[0] : 0);
+        uint4 kval = make_uint4(0u, 0u, 0u, 0u), vval = kval;
+        if (f) { kval = kbase[size_t(t) * 16 + col]; vval = vbase[size_t(t) * 16 + col]; }
+        done += s_wcnt[0] + s_wcnt[1];
+        __syncthreads();
+        if (f && dst != t) { kbase[size_t(dst) * 16 + col] = kval; vbase[size_t(dst) * 16 + col] = vval; }
+        __syncthreads();
+    }
+}
+
+template <bool kFill>
 __global__ void __launch_bounds__(kPlanThreads)
 compact_plan_kernel(int Hk, int max_sent, const int64_t* slab_off, const int32_t* cap, const uint8_t* keep,
-                    int32_t* sent_off, int32_t* sent_id, int32_t* n_sent, int32_t* kv_len, Header* hdr,
-                    int32_t* cp_nseg, uint32_t* cp_loaded, int32_t* cp_nruns, int32_t* cp_run_src,
-                    int32_t* cp_run_dst) {
+                    const uint8_t* tok_keep, uint4* K, uint4* V, int32_t* sent_off, int32_t* sent_id, int32_t* n_sent,
+                    int32_t* kv_len, Header* hdr, int32_t* cp_nseg, uint32_t* cp_loaded, int32_t* cp_nruns,
+                    int32_t* cp_run_src, int32_t* cp_run_dst, int32_t* cp_part) {
     __shared__ int wsum[kPlanThreads / 32][3];
     __shared__ int s_bad;
+    __shared__ int s_npart, s_part[kMaxPartial][3], s_pos[64], s_wcnt[2];
     // the move kernel is launched as a programmatic dependent: let its CTAs set themselves up while this grid runs
     pdl_trigger();
     pdl_wait();                                          // inputs may come from the kernel before
@@ -72,7 +107,12 @@ compact_plan_kernel(int Hk, int max_sent, const int64_t* slab_off, const int32_t
     int32_t* run_dst = cp_run_dst + size_t(slab) * (max_sent + 1);
     const int S = n_sent[slab];
     const int capb = cap[b];
+    const size_t row0 = slab_row0(slab_off, cap, Hk, b, slab % Hk);
+    const uint8_t* tk = kFill ? tok_keep + row0 : nullptr;
+    int32_t* part = cp_part + size_t(slab) * (1 + 3 * kMaxPartial);
     if (tid == 0) {
+        s_npart = 0;
+        if (kFill) part[0] = 0;
         s_bad = (S < 0 || S > max_sent) ? 1 : 0;
         cp_loaded[2 * slab] = 0u;
         cp_loaded[2 * slab + 1] = 0u;
@@ -87,21 +127,30 @@ compact_plan_kernel(int Hk, int max_sent, const int64_t* slab_off, const int32_t
     int prev_alive_carry = 0;
     for (int base = 0; base < S; base += kPlanThreads) {
         const int i = base + tid;
-        int b_i = 0, e_i = 0, id_i = -1, alive = 0;
+        int b_i = 0, e_i = 0, id_i = -1, alive = 0, klen = 0;
         if (i < S) {
             b_i = so[i]; e_i = so[i + 1]; id_i = sid[i];
             if (b_i < 0 || e_i < b_i || e_i > capb || (i == 0 && b_i != 0)) atomicOr(&s_bad, 1);
-            else alive = (kp[i] != 0 && e_i > b_i) ? 1 : 0;
+            else if (kp[i] != 0 && e_i > b_i) {
+                klen = e_i - b_i;
+                if (kFill && kp[i] == 2) {               // partly kept: count its survivors
+                    klen = 0;
+                    for (int t = b_i; t < e_i; ++t) klen += tk[t] != 0 ? 1 : 0;
+                }
+                alive = klen > 0 ? (klen < e_i - b_i ? 3 : 1) : 0;   // bit 1: rows are missing behind this sentence
+            }
         }
-        // does the previous sentence also survive?  (adjacent survivors form one run)
+        // does the previous sentence also survive, whole?  (adjacent whole survivors form one run; a partly
+        // kept sentence can end a run but nothing can follow it in the same run)
         int prev_alive = __shfl_up_sync(0xffffffffu, alive, 1);
         __shared__ int s_last[kPlanThreads / 32];
         if ((tid & 31) == 31) s_last[tid >> 5] = alive;
         __syncthreads();
         if ((tid & 31) == 0) prev_alive = (tid == 0) ? prev_alive_carry : s_last[(tid >> 5) - 1];
         const int last_alive = s_last[kPlanThreads / 32 - 1];
-        const int klen = alive ? (e_i - b_i) : 0;
-        const int start = (alive && !prev_alive) ? 1 : 0;
+        const int start = (alive && prev_alive != 1) ? 1 : 0;
+        const int partial = alive == 3;
+        alive = alive ? 1 : 0;
         int x_len, x_cnt, x_run, tot[3];
         block_scan3(klen, alive, start, x_len, x_cnt, x_run, tot, wsum);   // syncs: old values are all read
         if (alive) {
@@ -110,6 +159,11 @@ compact_plan_kernel(int Hk, int max_sent, const int64_t* slab_off, const int32_t
             if (start) {
                 run_src[c_run + x_run] = b_i;
                 run_dst[c_run + x_run] = c_len + x_len;
+            }
+            if (kFill && partial) {
+                const int q = atomicAdd(&s_npart, 1);
+                if (q < kMaxPartial) { s_part[q][0] = b_i; s_part[q][1] = e_i; s_part[q][2] = c_len + x_len; }
+                else atomicOr(&s_bad, 1);
             }
         }
         c_len += tot[0]; c_cnt += tot[1]; c_run += tot[2];
@@ -130,6 +184,43 @@ compact_plan_kernel(int Hk, int max_sent, const int64_t* slab_off, const int32_t
         kv_len[slab] = c_len;
         cp_nruns[slab] = c_run;
         cp_nseg[slab] = (c_len + kSegRows - 1) / kSegRows;
+    }
+    if (kFill) {
+        __syncthreads();
+        const int np = s_npart;
+        if (tid < np * 3) part[1 + tid] = s_part[tid / 3][tid % 3];
+        if (tid == 0) part[0] = np;
+        for (int q = 0; q < np; ++q) {                     // uniform over the CTA
+            pack_rows(K + row0 * 16, V + row0 * 16, tk, s_part[q][0], s_part[q][1], s_pos, s_wcnt);
+        }
+    }
+}
+
+// index_map entries of the partly kept sentences: destination token dst + k came from the k-th flagged token.
+__global__ void __launch_bounds__(64)
+compact_fill_index_kernel(int Hk, const int64_t* slab_off, const int32_t* cap, const uint8_t* tok_keep,
+                          int32_t* index_map, const int32_t* cp_part) {
+    __shared__ int s_wcnt[2];
+    const int slab = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    pdl_trigger();
+    pdl_wait();                                          // after the move kernel, which wrote the run-based entries
+    const int32_t* part = cp_part + size_t(slab) * (1 + 3 * kMaxPartial);
+    const int np = min(part[0], kMaxPartial);
+    const size_t row0 = slab_row0(slab_off, cap, Hk, slab / Hk, slab % Hk);
+    for (int q = 0; q < np; ++q) {
+        const int pb = part[1 + 3 * q], pe = part[2 + 3 * q], dst = part[3 + 3 * q];
+        int done = 0;
+        for (int cb = pb; cb < pe; cb += 64) {
+            const int t = cb + tid;
+            const int f = (t < pe) ? (tok_keep[row0 + t] != 0) : 0;
+            const unsigned m = __ballot_sync(0xffffffffu, f);
+            if (lane == 0) s_wcnt[warp] = __popc(m);
+            __syncthreads();
+            const int pos = done + __popc(m & ((1u << lane) - 1u)) + (warp ? s_wcnt[0] : 0);
+            if (f) index_map[row0 + dst + pos] = t;
+            done += s_wcnt[0] + s_wcnt[1];
+            __syncthreads();
+        }
     }
 }
 
@@ -256,9 +347,9 @@ compact_move_kernel(int n_slabs, int Hk, int max_sent, const int64_t* slab_off, 
 
 using namespace skipkv;
 
-extern "C" int skipkv_compact(const skipkv_shape* shape, void* K, void* V, const uint8_t* keep,
-                              int32_t* sent_off, int32_t* sent_id, int32_t* n_sent, int32_t* kv_len,
-                              int32_t* index_map, void* ws, void* stream) {
+static int compact_impl(const skipkv_shape* shape, void* K, void* V, const uint8_t* keep, const uint8_t* tok_keep,
+                        int32_t* sent_off, int32_t* sent_id, int32_t* n_sent, int32_t* kv_len, int32_t* index_map,
+                        void* ws, void* stream) {
     if (int rc = check_shape(shape)) return rc;
     if (!K || !V || !keep || !sent_off || !sent_id || !n_sent || !kv_len) return SKIPKV_ERR_INVALID_ARG;
     if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255)) return SKIPKV_ERR_WORKSPACE;
@@ -273,9 +364,12 @@ extern "C" int skipkv_compact(const skipkv_shape* shape, void* K, void* V, const
     int32_t* run_dst = reinterpret_cast<int32_t*>(w + L.cp_run_dst);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
 
-    SKIPKV_CUDA(launch_dependent(compact_plan_kernel, dim3(L.slabs), dim3(kPlanThreads), 0, st, int(shape->n_kv_heads),
-                                 int(shape->max_sent), shape->slab_off, shape->cap, keep, sent_off, sent_id, n_sent, kv_len,
-                                 hdr, nseg, loaded, nruns, run_src, run_dst));
+    int32_t* part = reinterpret_cast<int32_t*>(w + L.cp_part);
+    auto plan = tok_keep ? compact_plan_kernel<true> : compact_plan_kernel<false>;
+    SKIPKV_CUDA(launch_dependent(plan, dim3(L.slabs), dim3(kPlanThreads), 0, st, int(shape->n_kv_heads),
+                                 int(shape->max_sent), shape->slab_off, shape->cap, keep, tok_keep, static_cast<uint4*>(K),
+                                 static_cast<uint4*>(V), sent_off, sent_id, n_sent, kv_len, hdr, nseg, loaded, nruns,
+                                 run_src, run_dst, part));
 
     // set on every call: the attribute belongs to the current device's context, which a cached flag would not track
     SKIPKV_CUDA(cudaFuncSetAttribute(compact_move_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSegBytes));
@@ -283,5 +377,21 @@ extern "C" int skipkv_compact(const skipkv_shape* shape, void* K, void* V, const
                                  int(L.slabs), int(shape->n_kv_heads), int(shape->max_sent), shape->slab_off, shape->cap,
                                  static_cast<__nv_bfloat16*>(K), static_cast<__nv_bfloat16*>(V), index_map, hdr, nseg, loaded,
                                  nruns, run_src, run_dst));
+    if (tok_keep && index_map)
+        SKIPKV_CUDA(launch_dependent(compact_fill_index_kernel, dim3(L.slabs), dim3(64), 0, st, int(shape->n_kv_heads),
+                                     shape->slab_off, shape->cap, tok_keep, index_map, static_cast<const int32_t*>(part)));
     return SKIPKV_OK;
+}
+
+extern "C" int skipkv_compact(const skipkv_shape* shape, void* K, void* V, const uint8_t* keep,
+                              int32_t* sent_off, int32_t* sent_id, int32_t* n_sent, int32_t* kv_len,
+                              int32_t* index_map, void* ws, void* stream) {
+    return compact_impl(shape, K, V, keep, nullptr, sent_off, sent_id, n_sent, kv_len, index_map, ws, stream);
+}
+
+extern "C" int skipkv_compact_fill(const skipkv_shape* shape, void* K, void* V, const uint8_t* keep,
+                                   const uint8_t* tok_keep, int32_t* sent_off, int32_t* sent_id, int32_t* n_sent,
+                                   int32_t* kv_len, int32_t* index_map, void* ws, void* stream) {
+    if (!tok_keep) return SKIPKV_ERR_INVALID_ARG;
+    return compact_impl(shape, K, V, keep, tok_keep, sent_off, sent_id, n_sent, kv_len, index_map, ws, stream);
 }

@@ -9,6 +9,7 @@
 // prefix-summed in rank order, and a sentence survives iff its inclusive running total is
 // within the budget.  Because lengths are non-negative the running total is monotone, so this
 // is exactly "the longest rank prefix that fits; stop at the first sentence that does not".
+// skipkv_select_fill then lets that first sentence keep its most important tokens, so that exactly B survive.
 #include "common.cuh"
 
 namespace skipkv {
@@ -43,14 +44,26 @@ __device__ __forceinline__ uint32_t block_excl(uint32_t v, uint32_t* wsum, uint3
     return base + inc - v;
 }
 
+// Exactly-B retention: where tok_keep is non-null the first sentence that does not fit keeps its `slack` tokens of
+// largest importance (equal values: the earlier token), flagged in tok_keep (one byte per cache row), and gets
+// keep = 2.  tok_imp is indexed by cache row when from_rows is set, else [slab][max_cap].
+struct FillArgs {
+    const float* tok_imp;
+    uint8_t* tok_keep;
+    const int64_t* slab_off;
+    const int32_t* cap;
+    int Hk, max_cap, from_rows;
+};
+
 __global__ void __launch_bounds__(kSelThreads)
 select_kernel(int max_sent, int P, int budget, int protect_tail, const float* sent_score, const int32_t* sent_off,
               const int32_t* n_sent, uint8_t* keep, int32_t* kept_idx, int32_t* n_kept, int32_t* new_len,
-              uint32_t* status) {
+              FillArgs fill, uint32_t* status) {
     extern __shared__ __align__(16) uint8_t sel_smem[];
     uint64_t* keys = reinterpret_cast<uint64_t*>(sel_smem);             // [P]
     uint8_t* flags = reinterpret_cast<uint8_t*>(keys + P);             // [P] keep flag by sentence index
     __shared__ uint32_t wsum[kSelThreads / 32];
+    __shared__ int s_cut, s_slack;
     pdl_trigger();
     pdl_wait();                                          // inputs may come from the kernel before
     const int slab = blockIdx.x, tid = threadIdx.x;
@@ -88,6 +101,7 @@ select_kernel(int max_sent, int P, int budget, int protect_tail, const float* se
         keys[i] = k;
         flags[i] = 0;
     }
+    if (tid == 0) { s_cut = -1; s_slack = 0; }
     __syncthreads();
     // bitonic sort, ascending.  Thread p of a pass owns the compare-exchange pair (i, i | j) with
     // i = ((p & ~(j-1)) << 1) | (p & (j-1)).  For j <= 32 the 32 pairs of a warp stay inside the warp's own
@@ -116,21 +130,43 @@ select_kernel(int max_sent, int P, int budget, int protect_tail, const float* se
     uint32_t kept_tokens = 0;
     for (int r = r0; r < r1; ++r) {
         const int i = int(keys[r] & 0x7fffffffu);
+        const uint32_t before = run;
         run += uint32_t(so[i + 1] - so[i]);
         if (run <= uint32_t(budget)) { flags[i] = 1; kept_tokens = run; }
+        else if (fill.tok_keep && before < uint32_t(budget)) { s_cut = i; s_slack = budget - int(before); }  // one rank only
     }
     __syncthreads();
+    if (fill.tok_keep && s_cut >= 0) {
+        const int c = s_cut, slack = s_slack;
+        const int cb = so[c], len = so[c + 1] - cb;
+        const int b = slab / fill.Hk, h = slab % fill.Hk;
+        const size_t row0 = slab_row0(fill.slab_off, fill.cap, fill.Hk, b, h);
+        const float* imp = fill.from_rows ? fill.tok_imp + row0 + cb : fill.tok_imp + size_t(slab) * fill.max_cap + cb;
+        uint8_t* tk = fill.tok_keep + row0 + cb;
+        for (int t = tid; t < len; t += kSelThreads) {   // rank by counting: tokens that come before t in the order
+            const float mine = imp[t];
+            int rank = 0;
+            for (int u = 0; u < len; ++u) {
+                const float other = __ldg(imp + u);
+                rank += (other > mine || (other == mine && u < t)) ? 1 : 0;
+            }
+            tk[t] = rank < slack ? 1 : 0;
+        }
+        if (tid == 0) flags[c] = 2;
+        __syncthreads();
+    }
+    const bool filled = fill.tok_keep && s_cut >= 0;
     // outputs in sentence-index order
     const int per_i = (max(S, 1) + kSelThreads - 1) / kSelThreads;
     const int i0 = tid * per_i, i1 = min(i0 + per_i, S);
     uint32_t cnt = 0;
-    for (int i = i0; i < i1; ++i) cnt += flags[i];
+    for (int i = i0; i < i1; ++i) cnt += flags[i] ? 1u : 0u;
     uint32_t nk;
     uint32_t pos = block_excl(cnt, wsum, nk);
     for (int i = i0; i < i1; ++i) {
         kp[i] = flags[i];
         if (flags[i] && ki) ki[pos] = i;
-        pos += flags[i];
+        pos += flags[i] ? 1u : 0u;
     }
     for (int i = S + tid; i < max_sent; i += kSelThreads) kp[i] = 0;
     if (ki) for (int i = int(nk) + tid; i < max_sent; i += kSelThreads) ki[i] = -1;
@@ -145,7 +181,7 @@ select_kernel(int max_sent, int P, int budget, int protect_tail, const float* se
         uint32_t mm = 0;
         for (int w = 0; w < kSelThreads / 32; ++w) mm = max(mm, wsum[w]);
         if (n_kept) n_kept[slab] = int(nk);
-        if (new_len) new_len[slab] = int(mm);
+        if (new_len) new_len[slab] = filled ? budget : int(mm);
     }
 }
 
@@ -153,9 +189,9 @@ select_kernel(int max_sent, int P, int budget, int protect_tail, const float* se
 
 using namespace skipkv;
 
-extern "C" int skipkv_select(const skipkv_shape* shape, const skipkv_params* params, const float* sent_score,
-                             const int32_t* sent_off, const int32_t* n_sent, uint8_t* keep, int32_t* kept_idx,
-                             int32_t* n_kept, int32_t* new_len, void* ws, void* stream) {
+static int select_impl(const skipkv_shape* shape, const skipkv_params* params, const float* sent_score,
+                       const int32_t* sent_off, const int32_t* n_sent, uint8_t* keep, int32_t* kept_idx,
+                       int32_t* n_kept, int32_t* new_len, FillArgs fill, void* ws, void* stream) {
     if (int rc = check_shape(shape)) return rc;
     if (!params || !sent_score || !sent_off || !n_sent || !keep) return SKIPKV_ERR_INVALID_ARG;
     if (params->budget < 0 || params->protect_tail < 0) return SKIPKV_ERR_INVALID_ARG;
@@ -169,6 +205,28 @@ extern "C" int skipkv_select(const skipkv_shape* shape, const skipkv_params* par
     const int slabs = shape->batch * shape->n_kv_heads;
     SKIPKV_CUDA(launch_dependent(select_kernel, dim3(slabs), dim3(kSelThreads), smem, static_cast<cudaStream_t>(stream),
                                  shape->max_sent, P, params->budget, params->protect_tail, sent_score, sent_off, n_sent, keep,
-                                 kept_idx, n_kept, new_len, &static_cast<Header*>(ws)->status));
+                                 kept_idx, n_kept, new_len, fill, &static_cast<Header*>(ws)->status));
     return SKIPKV_OK;
+}
+
+extern "C" int skipkv_select(const skipkv_shape* shape, const skipkv_params* params, const float* sent_score,
+                             const int32_t* sent_off, const int32_t* n_sent, uint8_t* keep, int32_t* kept_idx,
+                             int32_t* n_kept, int32_t* new_len, void* ws, void* stream) {
+    return select_impl(shape, params, sent_score, sent_off, n_sent, keep, kept_idx, n_kept, new_len, FillArgs{}, ws,
+                       stream);
+}
+
+extern "C" int skipkv_select_fill(const skipkv_shape* shape, const skipkv_params* params, const float* sent_score,
+                                  const float* tok_imp, const int32_t* sent_off, const int32_t* n_sent, uint8_t* keep,
+                                  uint8_t* tok_keep, int32_t* kept_idx, int32_t* n_kept, int32_t* new_len, void* ws,
+                                  void* stream) {
+    if (!tok_keep) return SKIPKV_ERR_INVALID_ARG;
+    if (int rc = check_shape(shape)) return rc;
+    if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255)) return SKIPKV_ERR_WORKSPACE;
+    FillArgs fill{};
+    fill.tok_keep = tok_keep;
+    fill.slab_off = shape->slab_off; fill.cap = shape->cap; fill.Hk = shape->n_kv_heads; fill.max_cap = shape->max_cap;
+    if (tok_imp) { fill.tok_imp = tok_imp; fill.from_rows = 1; }
+    else { fill.tok_imp = reinterpret_cast<const float*>(static_cast<uint8_t*>(ws) + make_layout(*shape).sc_tokimp); }
+    return select_impl(shape, params, sent_score, sent_off, n_sent, keep, kept_idx, n_kept, new_len, fill, ws, stream);
 }

@@ -117,3 +117,44 @@ def test_qwen14b_shape_sampled_slabs():
     8192) at two sequences: one slab of each recomputed."""
     cfg = W.config(5, batch=2)
     run_case(cfg, [(0, 1), (1, 6)])
+
+
+def test_llama8b_32k_batch10_exactly_b_sampled_slabs():
+    """The headline workload through the exactly-B variants: every slab ends at the budget; three slabs are
+    recomputed by the oracle from the GPU's own scores and importances (selection, token flags, moved rows,
+    index map, tables: bit-exact)."""
+    from paper_2512_07993_b200 import build, binding as B
+    build.build()
+    cfg = W.config(2)
+    L = W.make_layer(cfg)
+    D = B.DeviceLayer(L)
+    tok_keep = torch.zeros(D.K.shape[0], dtype=torch.uint8, device="cuda")
+    D.score()
+    B.skipkv_select_fill(D.shape, D.params, D.sent_score, D.tok_imp, D.sent_off, D.n_sent, D.keep, tok_keep, D.kept_idx,
+                         D.n_kept, D.new_len, D.ws)
+    torch.cuda.synchronize()
+    sc, tok = D.sent_score.cpu().numpy(), D.tok_imp.cpu().numpy()
+    keep, tk = D.keep.cpu().numpy(), tok_keep.cpu().numpy()
+    B.skipkv_compact_fill(D.shape, D.K, D.V, D.keep, tok_keep, D.sent_off, D.sent_id, D.n_sent, D.kv_len, D.index_map, D.ws)
+    torch.cuda.synchronize()
+    assert D.status() == 0
+    kv_after = D.kv_len.cpu().numpy()
+    assert (kv_after == cfg.budget).all() and (D.new_len.cpu().numpy() == cfg.budget).all()
+    assert ((keep == 2).sum(axis=-1) <= 1).all()
+    Kb, Vb = W.bf16_bits(L["K"]), W.bf16_bits(L["V"])
+    Kg, Vg, imap = W.bf16_bits(D.K.cpu()), W.bf16_bits(D.V.cpu()), D.index_map.cpu().numpy()
+    so_after, ns_after = D.sent_off.cpu().numpy(), D.n_sent.cpu().numpy()
+    for (b, h) in [(0, 0), (4, 5), (9, 7)]:
+        rows = W.slab_rows(L, b, h)
+        N, S = int(L["kv_len"][b, h]), int(L["n_sent"][b, h])
+        off = L["sent_off"][b, h, :S + 1]
+        k_ref, t_ref, nl = oracle.select_fill(sc[b, h, :S], off, tok[rows][:N], cfg.budget, cfg.window)
+        assert np.array_equal(keep[b, h, :S], k_ref) and nl == cfg.budget
+        for c in np.nonzero(k_ref == 2)[0]:
+            assert np.array_equal(tk[rows][off[c]:off[c + 1]], t_ref[off[c]:off[c + 1]])
+        Ko, Vo, im, nso, nsid = oracle.compact_tokens(Kb[rows][:N], Vb[rows][:N], t_ref, off, L["sent_id"][b, h, :S])
+        n = len(im)
+        assert n == cfg.budget
+        assert np.array_equal(Kg[rows][:n], Ko) and np.array_equal(Vg[rows][:n], Vo)
+        assert np.array_equal(imap[rows][:n], im)
+        assert int(ns_after[b, h]) == len(nsid) and np.array_equal(so_after[b, h, :len(nso)], nso)
