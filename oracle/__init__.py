@@ -239,6 +239,19 @@ def compact_tokens(K_bits, V_bits, tok_keep, sent_off, sent_id):
             np.asarray(new_id, np.int32))
 
 
+# ------------------------------------------------------------------ token-level redundancy
+def token_redundancy(K_bits, eps=1e-6):
+    """O14  Token redundancy at token granularity (Section 4.1, token-redundancy equation):
+    Kbar_t = K_t / (|K_t|_2 + eps), G = Kbar Kbar^T, R = column mean of the row softmax of G with the
+    diagonal excluded -- O2 with every token its own sentence, followed by O3.  K_bits uint16 [N, d].
+    Returns R float64 [N]."""
+    K_bits = _c(K_bits, np.uint16)
+    N = K_bits.shape[0]
+    _, kbar = pool(K_bits, np.arange(N + 1, dtype=np.int32), np.zeros(N, np.float64), eps)
+    _, red, _ = gram_terms(kbar, 2.0)
+    return red
+
+
 # ------------------------------------------------------------------ batch drivers
 def score_batch(shape, K_bits, qwin_bits, kv_len, sent_off, n_sent, sigma, tau, eps, want_tok_imp=False):
     """shape: dict(batch,Hq,Hk,d,alpha,max_sent,slab_off,cap).  Returns dict of arrays."""

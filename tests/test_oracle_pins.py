@@ -606,6 +606,30 @@ def test_o13_hand_example():
     assert np.array_equal(unbits(Ko)[:, 0], [0, 2, 4, 12, 16])
 
 
+# ------------------------------------------------------------------ O14 token-level redundancy
+def test_o14_closed_form_and_library():
+    e = np.eye(4)
+    # keys 0 and 1 point the same way (different lengths), key 2 is orthogonal: the 3-sentence closed form of O3
+    R = oracle.token_redundancy(bits(np.stack([2 * e[0], 8 * e[0], 4 * e[1]])), eps=0.0)
+    E = math.e
+    assert np.allclose(R, [(E / (E + 1) + 0.5) / 3, (E / (E + 1) + 0.5) / 3, (2 / (E + 1)) / 3], atol=1e-15)
+    assert oracle.token_redundancy(bits(e[:1]))[0] == 0.0            # a single token has nothing to repeat
+    N, d = 37, 16
+    Kb = bits(rng.standard_normal((N, d)))
+    R = oracle.token_redundancy(Kb)
+    Kd = torch.from_numpy(unbits(Kb))
+    Kn = Kd / (Kd.norm(dim=1, keepdim=True) + 1e-6)
+    Gt = (Kn @ Kn.T).masked_fill(torch.eye(N, dtype=torch.bool), float("-inf"))
+    ref = torch.softmax(Gt, dim=1).sum(dim=0) / N
+    assert np.allclose(R, ref.numpy(), rtol=1e-12) and abs(R.sum() - 1.0) < 1e-13
+    # scaling a key changes nothing (cosine), repeating it raises its redundancy above an unrelated key's
+    K2 = unbits(Kb).copy(); K2[5] *= 4.0
+    assert np.allclose(oracle.token_redundancy(bits(K2)), R, rtol=1e-6)
+    K3 = unbits(Kb).copy(); K3[7] = K3[3]
+    R3 = oracle.token_redundancy(bits(K3))
+    assert R3[3] > R[3] and R3[7] > np.median(R3)
+
+
 def test_batch_drivers_match_slab_functions():
     cfg = W.config(0)
     L = W.make_layer(cfg)
