@@ -12,7 +12,8 @@
  *   skipkv_steer        steering-vector add on the hidden state
  * and, beside them, the generation-space lookup table of the sentence penalty (skipkv_table_step)
  * with the score variant that reads it (skipkv_score_table), and the variants of select and compact that
- * retain exactly B tokens (skipkv_select_fill, skipkv_compact_fill).
+ * retain exactly B tokens (skipkv_select_fill, skipkv_compact_fill), and the redundancy term over single
+ * tokens (skipkv_token_redundancy).
  *
  * Conventions
  *   - Every pointer marked "device" is a CUDA device pointer; "host" is ordinary memory.
@@ -253,6 +254,21 @@ int skipkv_select_fill(const skipkv_shape* shape, const skipkv_params* params, c
 int skipkv_compact_fill(const skipkv_shape* shape, void* K, void* V, const uint8_t* keep,
                         const uint8_t* tok_keep, int32_t* sent_off, int32_t* sent_id, int32_t* n_sent,
                         int32_t* kv_len, int32_t* index_map, void* ws, void* stream);
+
+/*
+ * skipkv_token_redundancy -- the token-redundancy equation of Section 4.1 at token granularity: per slab
+ * with N = kv_len[b][h] live rows,
+ *   Kbar_t = K_t / (|K_t|_2 + eps),   G = Kbar Kbar^T  (N x N),
+ *   tok_red[i] = (1/N) sum_{j != i} exp(G_ji) / sum_{k != j} exp(G_jk)
+ * (row softmax with the diagonal excluded, then the column mean; the values of a slab sum to 1; N = 1 gives
+ * 0).  This is what skipkv_score computes over pooled sentence keys, taken over the slab's own key rows:
+ * the cost grows with N^2, so it is meant for caches near the budget (N about B + the decode interval).
+ * K: device bf16 cache (read only).  tok_red: device fp32, one value per cache row with the row indexing of
+ * K; rows at and beyond kv_len are not written.  params->eps is used; shape->total_rows must be the exact
+ * row count of K.  Launch behaviour as skipkv_score.
+ */
+int skipkv_token_redundancy(const skipkv_shape* shape, const skipkv_params* params, const void* K,
+                            const int32_t* kv_len, float* tok_red, void* ws, void* stream);
 
 /*
  * skipkv_decode_attn_static -- skipkv_decode_attn for callers that cannot allocate device

@@ -22,7 +22,7 @@ ERRORS = {-1: "SKIPKV_ERR_INVALID_ARG", -2: "SKIPKV_ERR_UNSUPPORTED", -3: "SKIPK
 SYMBOLS = ["skipkv_workspace_bytes", "skipkv_workspace_init", "skipkv_status", "skipkv_last_cuda_error",
            "skipkv_score", "skipkv_select", "skipkv_compact", "skipkv_decode_attn", "skipkv_steer",
            "skipkv_append", "skipkv_decode_attn_static", "skipkv_table_step", "skipkv_score_table",
-           "skipkv_select_fill", "skipkv_compact_fill"]
+           "skipkv_select_fill", "skipkv_compact_fill", "skipkv_token_redundancy"]
 
 
 class SkipKVError(RuntimeError):
@@ -196,6 +196,12 @@ def skipkv_compact_fill(shape, K, V, keep, tok_keep, sent_off, sent_id, n_sent, 
                                      _ptr(sent_off, torch.int32), _ptr(sent_id, torch.int32),
                                      _ptr(n_sent, torch.int32), _ptr(kv_len, torch.int32),
                                      _ptr(index_map, torch.int32), _ptr(ws), _stream(stream)), "skipkv_compact_fill")
+
+
+def skipkv_token_redundancy(shape, params, K, kv_len, tok_red, ws, stream=None) -> None:
+    _check(lib().skipkv_token_redundancy(C.byref(shape), C.byref(params), _ptr(K, torch.bfloat16),
+                                         _ptr(kv_len, torch.int32), _ptr(tok_red, torch.float32), _ptr(ws),
+                                         _stream(stream)), "skipkv_token_redundancy")
 
 
 def skipkv_decode_attn_static(shape, q, K, V, kv_len, out, hidden, steer_vec, alpha, flag, status=None,

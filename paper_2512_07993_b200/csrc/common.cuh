@@ -40,6 +40,8 @@ struct WsLayout {
     size_t sc_vbar_lo;     // bf16   [slabs][max_sent][128]  and the rounding remainder
     size_t sc_z;           // float  [slabs][max_sent]
     size_t cp_part;        // int32  [slabs][1 + 3*kMaxPartial]  partly kept sentences: count, then (begin, end, dst)
+    size_t tr_inv;         // float  [slabs][max_cap]  token redundancy: 1 / (|K_t| + eps)
+    size_t tr_z;           // float  [slabs][max_cap]  token redundancy: row sums of exp(G)
     size_t total;
     int slabs, group, qrows, dec_max_ctas;
     int sc_wb;             // window positions per query block: floor(128 / group)
@@ -78,6 +80,8 @@ inline WsLayout make_layout(const skipkv_shape& s) {
     L.sc_vbar_lo = take(slabs * ms * kHeadDim * 2);
     L.sc_z = take(slabs * ms * 4);
     L.cp_part = take(slabs * (1 + 3 * kMaxPartial) * 4);
+    L.tr_inv = take(slabs * size_t(s.max_cap > 0 ? s.max_cap : 1) * 4);
+    L.tr_z = take(slabs * size_t(s.max_cap > 0 ? s.max_cap : 1) * 4);
     L.total = o;
     return L;
 }

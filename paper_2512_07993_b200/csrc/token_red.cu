@@ -1,0 +1,304 @@
+// skipkv_token_redundancy: the token-redundancy term at TOKEN granularity (paper Section 4.1,
+// token-redundancy equation: R = mean(softmax(Kbar Kbar^T)) with Kbar = K / (||K||_2 + eps)), an
+// N' x N' Gram matrix per (sequence, KV head) slab over the slab's own key rows:
+//     G_ij  = K_i . K_j / ((|K_i| + eps)(|K_j| + eps))
+//     Z_j   = sum_{k != j} exp(G_jk)
+//     R_i   = (1/N') sum_{j != i} exp(G_ji) / Z_j
+// Three launches:
+//   token_norm_kernel      1 / (|K_t| + eps) of every live row (a warp per row);
+//   token_red_kernel<1>    row sums Z;
+//   token_red_kernel<2>    R.
+// The Gram kernels are persistent and warp-specialised: a work item is 128 rows i of one slab against
+// every block of 128 rows j of the same slab.  Warp 0 streams the bf16 key tiles straight from the cache
+// with tiled TMA loads (the i tile once per item, the j tiles through a ring), warp 1 issues one
+// 128 x 128 x 128 tcgen05.mma group per (i, j) block into one of two tensor-memory accumulators, and four
+// warps read the accumulators back, scale by the two inverse norms and exponentiate.  The products of bf16
+// keys are exact in fp32, so no operand is rounded: normalisation happens after the contraction.
+// One exponential per matrix element makes the special-function unit, not the tensor pipe, the limit.
+#include "tc.cuh"
+
+namespace skipkv {
+
+constexpr int kTrThreads = 6 * 32;
+constexpr int kTrStages = 4;                 // j tiles in flight
+constexpr float kTrLog2e = 1.4426950408889634f;
+
+struct TrCtl {
+    uint64_t afull, aempty, bfull[kTrStages], bempty[kTrStages], tfull[2], tempty[2];
+    uint32_t tmem_base;
+    int abort_flag;
+    uint32_t wsum[8];
+    float jn[2][128];                        // log2(e) / (|K_j| + eps) of the j block under an accumulator
+    float jz[2][128];                        // pass 2: 1 / Z_j
+};
+static size_t tr_smem_bytes(int slabs) { return 1024 + (1 + kTrStages) * size_t(kOpBytes) + sizeof(TrCtl) + size_t(slabs + 1) * 4; }
+
+__device__ __forceinline__ float tr_ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+__global__ void __launch_bounds__(256)
+token_norm_kernel(int Hk, int max_cap, const int64_t* slab_off, const int32_t* cap, const __nv_bfloat16* K,
+                  const int32_t* kv_len, float eps, float* inv_norm) {
+    const int slab = blockIdx.y, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    pdl_trigger();
+    pdl_wait();
+    const int len = min(max(kv_len[slab], 0), min(cap[slab / Hk], max_cap));
+    const int t0 = blockIdx.x * 64 + warp * 8;
+    if (t0 >= len) return;
+    const size_t row0 = slab_row0(slab_off, cap, Hk, slab / Hk, slab % Hk);
+    uint2 x[8];
+#pragma unroll
+    for (int r = 0; r < 8; ++r)
+        x[r] = (t0 + r < len) ? reinterpret_cast<const uint2*>(K + (row0 + t0 + r) * kHeadDim)[lane] : make_uint2(0u, 0u);
+#pragma unroll
+    for (int r = 0; r < 8; ++r) {
+        const float a = bf16lo(x[r].x), b = bf16hi(x[r].x), c = bf16lo(x[r].y), d = bf16hi(x[r].y);
+        float ss = a * a + b * b + c * c + d * d;
+#pragma unroll
+        for (int s = 16; s; s >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, s);
+        if (lane == 0 && t0 + r < len) inv_norm[size_t(slab) * max_cap + t0 + r] = 1.f / (sqrtf(ss) + eps);
+    }
+}
+
+__device__ __forceinline__ bool tr_wait(TrCtl* ctl, uint64_t* bar, uint32_t parity, uint32_t* status) {
+    if (mbar_try_wait(bar, parity)) return true;
+    for (uint32_t i = 0; i < (1u << 22); ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (i > 64) {
+            __nanosleep(64);
+            if ((i & 255) == 0 && *reinterpret_cast<volatile int*>(&ctl->abort_flag)) return false;
+        }
+    }
+    atomicOr(status, SKIPKV_STATUS_COPY_TIMEOUT);
+    *reinterpret_cast<volatile int*>(&ctl->abort_flag) = 1;
+    return false;
+}
+
+template <int kPass>
+__global__ void __launch_bounds__(kTrThreads, 1)
+token_red_kernel(const __grid_constant__ CUtensorMap mapK, int n_slabs, int Hk, int max_cap, const int64_t* slab_off,
+                 const int32_t* cap, const int32_t* kv_len, const float* inv_norm, float* z, float* tok_red,
+                 uint32_t* status) {
+    extern __shared__ uint8_t tr_smem_raw[];
+    const uint32_t raw = smem_u32(tr_smem_raw);
+    uint8_t* At = tr_smem_raw + (((raw + 1023u) & ~1023u) - raw);
+    uint8_t* Bt = At + kOpBytes;
+    TrCtl* ctl = reinterpret_cast<TrCtl*>(Bt + kTrStages * kOpBytes);
+    int* ipref = reinterpret_cast<int*>(ctl + 1);                                // [n_slabs + 1] prefix of i blocks
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int G = gridDim.x, cta = blockIdx.x;
+    auto len_of = [&](int s) { return min(max(kv_len[s], 0), min(cap[s / Hk], max_cap)); };
+    pdl_trigger();
+
+    if (tid == 0) {
+        mbar_init(&ctl->afull, 1);
+        mbar_init(&ctl->aempty, 1);
+        for (int s = 0; s < kTrStages; ++s) { mbar_init(&ctl->bfull[s], 1); mbar_init(&ctl->bempty[s], 1); }
+        for (int s = 0; s < 2; ++s) { mbar_init(&ctl->tfull[s], 1); mbar_init(&ctl->tempty[s], 4); }
+        ctl->abort_flag = 0;
+        mbar_fence_init();
+        tmap_prefetch(&mapK);
+    }
+    if (warp == 1) tmem_alloc(&ctl->tmem_base, 256);
+    pdl_wait();                                          // kv_len and the norms may come from the kernels before
+    {   // prefix of i blocks over slabs (block scan; every thread owns a contiguous block of slabs)
+        const int per = (n_slabs + kTrThreads - 1) / kTrThreads;
+        const int s0 = min(tid * per, n_slabs), s1 = min(s0 + per, n_slabs);
+        uint32_t local = 0;
+        for (int s = s0; s < s1; ++s) local += uint32_t((len_of(s) + 127) >> 7);
+        uint32_t inc = local;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const uint32_t x = __shfl_up_sync(0xffffffffu, inc, d);
+            if (lane >= d) inc += x;
+        }
+        if (lane == 31) ctl->wsum[warp] = inc;
+        tc_fence_before();
+        __syncthreads();                                 // also publishes barrier inits and the tmem address
+        tc_fence_after();
+        uint32_t base = 0;
+        for (int w = 0; w < warp; ++w) base += ctl->wsum[w];
+        uint32_t run = base + inc - local;
+        for (int s = s0; s < s1; ++s) {
+            ipref[s] = int(run);
+            run += uint32_t((len_of(s) + 127) >> 7);
+        }
+        if (tid == kTrThreads - 1) ipref[n_slabs] = int(run);
+        __syncthreads();
+    }
+    const uint32_t tmem_base = ctl->tmem_base;
+    const int n_items = ipref[n_slabs];
+    auto row0_of = [&](int s) { return int(slab_row0(slab_off, cap, Hk, s / Hk, s % Hk)); };
+
+    if (warp == 0) {
+        if (lane == 0) {
+            bool ok = true;
+            int slab = 0;
+            uint32_t bc = 0, ic = 0;                                // j blocks and items issued so far
+            for (int item = cta; item < n_items && ok; item += G, ++ic) {
+                while (ipref[slab + 1] <= item) ++slab;
+                const int NJ = (len_of(slab) + 127) >> 7, row0 = row0_of(slab);
+                const int i0 = (item - ipref[slab]) * 128;
+                if (ic > 0) ok = tr_wait(ctl, &ctl->aempty, (ic - 1) & 1u, status);
+                if (!ok) break;
+                mbar_expect_tx(&ctl->afull, kOpBytes);
+                tma_load_2d(At, &mapK, 0, row0 + i0, &ctl->afull);
+                tma_load_2d(At + kOpHalfBytes, &mapK, 64, row0 + i0, &ctl->afull);
+                for (int jb = 0; jb < NJ && ok; ++jb, ++bc) {
+                    const int s = bc % kTrStages;
+                    if (bc >= kTrStages) ok = tr_wait(ctl, &ctl->bempty[s], ((bc / kTrStages) - 1) & 1u, status);
+                    if (!ok) break;
+                    uint8_t* dst = Bt + size_t(s) * kOpBytes;
+                    mbar_expect_tx(&ctl->bfull[s], kOpBytes);
+                    tma_load_2d(dst, &mapK, 0, row0 + jb * 128, &ctl->bfull[s]);
+                    tma_load_2d(dst + kOpHalfBytes, &mapK, 64, row0 + jb * 128, &ctl->bfull[s]);
+                }
+            }
+            if (!ok) {                                   // let the copies in flight land before the CTA exits
+                mbar_wait(&ctl->afull, 0u, 1u << 16); mbar_wait(&ctl->afull, 1u, 1u << 16);
+                for (int s = 0; s < kTrStages; ++s) { mbar_wait(&ctl->bfull[s], 0u, 1u << 16); mbar_wait(&ctl->bfull[s], 1u, 1u << 16); }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            bool ok = true;
+            int slab = 0;
+            uint32_t bc = 0, ic = 0;
+            const uint32_t a = smem_u32(At);
+            for (int item = cta; item < n_items && ok; item += G, ++ic) {
+                while (ipref[slab + 1] <= item) ++slab;
+                const int NJ = (len_of(slab) + 127) >> 7;
+                ok = tr_wait(ctl, &ctl->afull, ic & 1u, status);
+                for (int jb = 0; jb < NJ && ok; ++jb, ++bc) {
+                    const int st = bc % kTrStages, s = bc & 1;
+                    ok = tr_wait(ctl, &ctl->bfull[st], (bc / kTrStages) & 1u, status);
+                    if (ok && bc >= 2) ok = tr_wait(ctl, &ctl->tempty[s], ((bc >> 1) - 1) & 1u, status);
+                    if (!ok) break;
+                    tc_fence_after();
+                    umma_tile_128x128x128(tmem_base + s * 128, a, smem_u32(Bt + size_t(st) * kOpBytes), false);
+                    umma_commit(&ctl->tfull[s]);
+                    umma_commit(&ctl->bempty[st]);
+                }
+                if (ok) umma_commit(&ctl->aempty);                   // every MMA that reads this i tile has completed
+            }
+        }
+    } else {
+        const int quarter = warp & 3, wt = tid - 64;
+        const uint32_t lane_addr = tmem_base + (uint32_t(quarter * 32) << 16);
+        bool ok = true;
+        int slab = 0;
+        uint32_t bc = 0;
+        for (int item = cta; item < n_items; item += G) {
+            while (ipref[slab + 1] <= item) ++slab;
+            const int S = len_of(slab), NJ = (S + 127) >> 7;
+            const size_t sbase = size_t(slab) * max_cap;
+            const int i0 = (item - ipref[slab]) * 128;
+            const int i = i0 + quarter * 32 + lane;
+            const float inv_i = (i < S) ? inv_norm[sbase + i] : 0.f;
+            float accum = 0.f;
+            for (int jb = 0; jb < NJ; ++jb, ++bc) {
+                const int s = bc & 1, j0 = jb * 128;
+                {
+                    const int j = j0 + wt;
+                    ctl->jn[s][wt] = (j < S) ? inv_norm[sbase + j] * kTrLog2e : 0.f;
+                    if (kPass == 2) {
+                        const float zz = (j < S) ? z[sbase + j] : 1.f;
+                        ctl->jz[s][wt] = (zz > 0.f) ? 1.f / zz : 0.f;
+                    }
+                    named_bar_sync(1, 128);
+                }
+                if (ok) {
+                    ok = tr_wait(ctl, &ctl->tfull[s], (bc >> 1) & 1u, status);
+                    ok = __all_sync(0xffffffffu, ok);
+                }
+                if (!ok) continue;                               // keeps the barrier pattern uniform
+                tc_fence_after();
+                const bool interior = (j0 + 128 <= S) && (j0 != i0);
+#pragma unroll 1
+                for (int ch = 0; ch < 4; ++ch) {
+                    float v[32];
+                    tmem_ld32(lane_addr + s * 128 + ch * 32, v);
+                    const float* jn = ctl->jn[s] + ch * 32;
+                    const float* jz = ctl->jz[s] + ch * 32;
+                    if (interior) {
+                        float e0 = 0.f, e1 = 0.f;
+#pragma unroll
+                        for (int jj = 0; jj < 32; jj += 2) {
+                            if (kPass == 1) {
+                                e0 += tr_ex2(v[jj] * inv_i * jn[jj]);
+                                e1 += tr_ex2(v[jj + 1] * inv_i * jn[jj + 1]);
+                            } else {
+                                e0 = fmaf(tr_ex2(v[jj] * inv_i * jn[jj]), jz[jj], e0);
+                                e1 = fmaf(tr_ex2(v[jj + 1] * inv_i * jn[jj + 1]), jz[jj + 1], e1);
+                            }
+                        }
+                        accum += e0 + e1;
+                    } else {
+#pragma unroll
+                        for (int jj = 0; jj < 32; ++jj) {
+                            const int j = j0 + ch * 32 + jj;
+                            if (j < S && j != i) {
+                                const float e = tr_ex2(v[jj] * inv_i * jn[jj]);
+                                if (kPass == 1) accum += e; else accum = fmaf(e, jz[jj], accum);
+                            }
+                        }
+                    }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&ctl->tempty[s]);
+            }
+            if (ok && i < S) {
+                if (kPass == 1) z[sbase + i] = accum;
+                else tok_red[size_t(row0_of(slab)) + i] = accum / float(S);
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, 256);
+    }
+}
+
+}  // namespace skipkv
+
+using namespace skipkv;
+
+extern "C" int skipkv_token_redundancy(const skipkv_shape* shape, const skipkv_params* params, const void* K,
+                                       const int32_t* kv_len, float* tok_red, void* ws, void* stream) {
+    if (int rc = check_shape(shape)) return rc;
+    if (!params || !K || !kv_len || !tok_red) return SKIPKV_ERR_INVALID_ARG;
+    if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255)) return SKIPKV_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(K) & 15) return SKIPKV_ERR_INVALID_ARG;
+    const WsLayout L = make_layout(*shape);
+    uint8_t* w = static_cast<uint8_t*>(ws);
+    uint32_t* status = &reinterpret_cast<Header*>(w + L.header)->status;
+    float* inv_norm = reinterpret_cast<float*>(w + L.tr_inv);
+    float* z = reinterpret_cast<float*>(w + L.tr_z);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    CUtensorMap mapK;
+    if (int rc = tmap_rows(&mapK, K, uint64_t(shape->total_rows), 128)) return rc;
+    const size_t smem = tr_smem_bytes(L.slabs);
+    if (smem > 227 * 1024) return SKIPKV_ERR_UNSUPPORTED;
+    const int Hk = shape->n_kv_heads;
+    SKIPKV_CUDA(launch_dependent(token_norm_kernel, dim3((shape->max_cap + 63) / 64, L.slabs), dim3(256), 0, st, Hk,
+                                 int(shape->max_cap), shape->slab_off, shape->cap, static_cast<const __nv_bfloat16*>(K),
+                                 kv_len, params->eps, inv_norm));
+    const long long max_items = (long long)L.slabs * ((shape->max_cap + 127) / 128);
+    int grid = num_sms();
+    if (max_items < grid) grid = int(max_items);
+    SKIPKV_CUDA(cudaFuncSetAttribute(token_red_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
+    SKIPKV_CUDA(cudaFuncSetAttribute(token_red_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
+    SKIPKV_CUDA(launch_dependent(token_red_kernel<1>, dim3(grid), dim3(kTrThreads), smem, st, mapK, int(L.slabs), Hk,
+                                 int(shape->max_cap), shape->slab_off, shape->cap, kv_len, static_cast<const float*>(inv_norm),
+                                 z, tok_red, status));
+    SKIPKV_CUDA(launch_dependent(token_red_kernel<2>, dim3(grid), dim3(kTrThreads), smem, st, mapK, int(L.slabs), Hk,
+                                 int(shape->max_cap), shape->slab_off, shape->cap, kv_len, static_cast<const float*>(inv_norm),
+                                 z, tok_red, status));
+    return SKIPKV_OK;
+}
