@@ -182,6 +182,76 @@ def run_reference(args, rank):
     print(json.dumps(line), flush=True)
 
 
+def time_extras(cfg, B, flush, clean, peaks, reps=10):
+    """CUDA-event times (median, L2 flushed before every call) of the entry points beside the main path."""
+    def timed(fn, before=lambda: None):
+        ts = []
+        for _ in range(reps):
+            before()
+            flush.fill_(1); clean.sum()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); fn(); e1.record()
+            torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1) * 1e3)
+        return statistics.median(ts[3:])
+
+    out = {}
+    dev = "cuda"
+    # lookup-table step: every sequence closes a sentence that is compared with n_prev earlier ones
+    bt, dm, mg, n_prev = cfg.batch, cfg.d_model, 2048, 1300
+    emb = torch.randn(bt, mg, dm, device=dev); emb /= emb.norm(dim=-1, keepdim=True)
+    acc = torch.zeros(bt, dm, device=dev); cnt = torch.zeros(bt, dtype=torch.int32, device=dev)
+    T = torch.zeros(bt, mg, device=dev); closed = torch.zeros(bt, dtype=torch.int32, device=dev)
+    h = torch.randn(bt, dm, device=dev).bfloat16(); flag = torch.ones(bt, dtype=torch.uint8, device=dev)
+    n = torch.empty(bt, dtype=torch.int32, device=dev)
+    us = timed(lambda: B.skipkv_table_step(bt, dm, mg, h, flag, acc, cnt, emb, n, closed, T, 0.95, 1e-6),
+               before=lambda: n.fill_(n_prev))
+    byt = bt * n_prev * dm * 4
+    out["table_step"] = {"us": us, "earlier_sentences": n_prev, "d_model": dm, "algorithmic_bytes": byt,
+                         "bound": "hbm", "achieved": byt / us / 1e3, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                         "frac": byt / us / 1e3 / peaks["hbm_gbs"]}
+    del emb
+    # exactly-B variants on one layer of the workload, beside the plain calls timed the same way
+    L = W.make_layer(cfg)
+    D = B.DeviceLayer(L)
+    tok_keep = torch.zeros(D.K.shape[0], dtype=torch.uint8, device=dev)
+    keys = ("K", "V", "sent_off", "sent_id", "n_sent", "kv_len")
+    pristine = {k: getattr(D, k).clone() for k in keys}
+    def restore():
+        for k, v in pristine.items():
+            getattr(D, k).copy_(v)
+    select_fill = lambda: B.skipkv_select_fill(D.shape, D.params, D.sent_score, D.tok_imp, D.sent_off, D.n_sent, D.keep,
+                                               tok_keep, D.kept_idx, D.n_kept, D.new_len, D.ws)
+    compact_fill = lambda: B.skipkv_compact_fill(D.shape, D.K, D.V, D.keep, tok_keep, D.sent_off, D.sent_id, D.n_sent,
+                                                 D.kv_len, D.index_map, D.ws)
+    D.score()
+    out["select_us"] = timed(D.select, restore)
+    out["select_fill_us"] = timed(select_fill, restore)
+    restore(); D.select()
+    out["compact_us"] = timed(D.compact, restore)
+    restore(); select_fill()
+    out["compact_fill_us"] = timed(compact_fill, restore)
+    D.status()
+    del D, pristine, tok_keep
+    torch.cuda.empty_cache()
+    # token-level redundancy at the steady-state length of a budgeted cache: budget + 128 rows per slab
+    n_tok = cfg.budget + 128
+    cfg_ss = W.config(0, batch=cfg.batch, n_q_heads=cfg.n_q_heads, n_kv_heads=cfg.n_kv_heads, window=cfg.window,
+                      d_model=cfg.d_model, budget=cfg.budget, ctx_lo=n_tok, ctx_hi=n_tok, sent_lo=cfg.sent_lo,
+                      sent_hi=cfg.sent_hi, seed=cfg.seed)
+    D = B.DeviceLayer(W.make_layer(cfg_ss))
+    red = torch.zeros(D.K.shape[0], dtype=torch.float32, device=dev)
+    us = timed(lambda: B.skipkv_token_redundancy(D.shape, D.params, D.K, D.kv_len, red, D.ws))
+    D.status()
+    elems = cfg.batch * cfg.n_kv_heads * float(n_tok) * n_tok * 2          # matrix elements over both passes
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    mufu_peak = sms * 16 * peaks.get("sm_max_mhz", 1965.0) * 1e6 / 1e12     # 16 special-function results per SM per clock
+    out["token_redundancy"] = {"us": us, "rows_per_slab": n_tok, "bound": "alu", "achieved": elems / us / 1e6,
+                               "peak": mufu_peak, "unit": "T exp/s", "frac": elems / us / 1e6 / mufu_peak,
+                               "tensor_tflops": elems * 256 / us / 1e6}
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -193,6 +263,9 @@ def main():
     ap.add_argument("--layers", type=int, default=4, help="layers (independent K/V buffers) each leg of a step runs over")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--extras", action="store_true",
+                    help="also time the entry points beside the main path (lookup table, exactly-B variants, "
+                         "token-level redundancy); reported under \"extras\", not part of `value`")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "skipkv" else args.warmup
 
@@ -360,6 +433,10 @@ def main():
                                 "decode_attn_us": legs_s["decode_attn"] / frac * 1e6,
                                 "sample": f"first {n_seq} of {cfg.batch} sequences ({frac:.3f} of the tokens), "
                                           "time scaled by token count"}
+    if args.extras and world == 1:
+        del Ds, D, pristine
+        torch.cuda.empty_cache()
+        line["extras"] = time_extras(cfg, B, flush, clean, peaks)
     if rank == 0:
         print(json.dumps(line), flush=True)
     if dist:

@@ -11,25 +11,28 @@
 // The Gram kernels are persistent and warp-specialised: a work item is 128 rows i of one slab against
 // every block of 128 rows j of the same slab.  Warp 0 streams the bf16 key tiles straight from the cache
 // with tiled TMA loads (the i tile once per item, the j tiles through a ring), warp 1 issues one
-// 128 x 128 x 128 tcgen05.mma group per (i, j) block into one of two tensor-memory accumulators, and four
-// warps read the accumulators back, scale by the two inverse norms and exponentiate.  The products of bf16
+// 128 x 128 x 128 tcgen05.mma group per (i, j) block into one of four tensor-memory accumulators, and four
+// warpgroups (one per accumulator, so that one's tensor-memory reads hide behind the others' arithmetic)
+// read the accumulators back, scale by the two inverse norms and exponentiate.  The products of bf16
 // keys are exact in fp32, so no operand is rounded: normalisation happens after the contraction.
 // One exponential per matrix element makes the special-function unit, not the tensor pipe, the limit.
 #include "tc.cuh"
 
 namespace skipkv {
 
-constexpr int kTrThreads = 6 * 32;
+constexpr int kTrGroups = 4;                 // epilogue warpgroups = tensor-memory accumulators of 128 columns
+constexpr int kTrThreads = (2 + 4 * kTrGroups) * 32;   // TMA warp, MMA warp, epilogue warpgroups
 constexpr int kTrStages = 4;                 // j tiles in flight
 constexpr float kTrLog2e = 1.4426950408889634f;
 
 struct TrCtl {
-    uint64_t afull, aempty, bfull[kTrStages], bempty[kTrStages], tfull[2], tempty[2];
+    uint64_t afull, aempty, bfull[kTrStages], bempty[kTrStages], tfull[kTrGroups], tempty[kTrGroups];
     uint32_t tmem_base;
     int abort_flag;
-    uint32_t wsum[8];
-    float jn[2][128];                        // log2(e) / (|K_j| + eps) of the j block under an accumulator
-    float jz[2][128];                        // pass 2: 1 / Z_j
+    uint32_t wsum[32];
+    alignas(16) float jn[kTrGroups][128];    // log2(e) / (|K_j| + eps) of the j block under an accumulator
+    alignas(16) float jz[kTrGroups][128];    // pass 2: 1 / Z_j
+    float part[2][kTrGroups - 1][128];       // the other warpgroups' shares of an item's row sums (by item parity)
 };
 static size_t tr_smem_bytes(int slabs) { return 1024 + (1 + kTrStages) * size_t(kOpBytes) + sizeof(TrCtl) + size_t(slabs + 1) * 4; }
 
@@ -97,12 +100,12 @@ token_red_kernel(const __grid_constant__ CUtensorMap mapK, int n_slabs, int Hk, 
         mbar_init(&ctl->afull, 1);
         mbar_init(&ctl->aempty, 1);
         for (int s = 0; s < kTrStages; ++s) { mbar_init(&ctl->bfull[s], 1); mbar_init(&ctl->bempty[s], 1); }
-        for (int s = 0; s < 2; ++s) { mbar_init(&ctl->tfull[s], 1); mbar_init(&ctl->tempty[s], 4); }
+        for (int s = 0; s < kTrGroups; ++s) { mbar_init(&ctl->tfull[s], 1); mbar_init(&ctl->tempty[s], 4); }
         ctl->abort_flag = 0;
         mbar_fence_init();
         tmap_prefetch(&mapK);
     }
-    if (warp == 1) tmem_alloc(&ctl->tmem_base, 256);
+    if (warp == 1) tmem_alloc(&ctl->tmem_base, 128 * kTrGroups);
     pdl_wait();                                          // kv_len and the norms may come from the kernels before
     {   // prefix of i blocks over slabs (block scan; every thread owns a contiguous block of slabs)
         const int per = (n_slabs + kTrThreads - 1) / kTrThreads;
@@ -173,9 +176,9 @@ token_red_kernel(const __grid_constant__ CUtensorMap mapK, int n_slabs, int Hk, 
                 const int NJ = (len_of(slab) + 127) >> 7;
                 ok = tr_wait(ctl, &ctl->afull, ic & 1u, status);
                 for (int jb = 0; jb < NJ && ok; ++jb, ++bc) {
-                    const int st = bc % kTrStages, s = bc & 1;
+                    const int st = bc % kTrStages, s = bc % kTrGroups;
                     ok = tr_wait(ctl, &ctl->bfull[st], (bc / kTrStages) & 1u, status);
-                    if (ok && bc >= 2) ok = tr_wait(ctl, &ctl->tempty[s], ((bc >> 1) - 1) & 1u, status);
+                    if (ok && bc >= kTrGroups) ok = tr_wait(ctl, &ctl->tempty[s], ((bc / kTrGroups) - 1) & 1u, status);
                     if (!ok) break;
                     tc_fence_after();
                     umma_tile_128x128x128(tmem_base + s * 128, a, smem_u32(Bt + size_t(st) * kOpBytes), false);
@@ -186,32 +189,37 @@ token_red_kernel(const __grid_constant__ CUtensorMap mapK, int n_slabs, int Hk, 
             }
         }
     } else {
-        const int quarter = warp & 3, wt = tid - 64;
-        const uint32_t lane_addr = tmem_base + (uint32_t(quarter * 32) << 16);
+        const int grp = (warp - 2) >> 2;                           // the accumulator this warpgroup drains
+        const int quarter = warp & 3, wt = (tid - 64) & 127;
+        const uint32_t lane_addr = tmem_base + (uint32_t(quarter * 32) << 16) + grp * 128;
+        float* jn_s = ctl->jn[grp];
+        float* jz_s = ctl->jz[grp];
         bool ok = true;
         int slab = 0;
-        uint32_t bc = 0;
-        for (int item = cta; item < n_items; item += G) {
+        uint32_t bc = 0, ic = 0;
+        for (int item = cta; item < n_items; item += G, ++ic) {
             while (ipref[slab + 1] <= item) ++slab;
             const int S = len_of(slab), NJ = (S + 127) >> 7;
             const size_t sbase = size_t(slab) * max_cap;
             const int i0 = (item - ipref[slab]) * 128;
-            const int i = i0 + quarter * 32 + lane;
+            const int row = quarter * 32 + lane;
+            const int i = i0 + row;
             const float inv_i = (i < S) ? inv_norm[sbase + i] : 0.f;
             float accum = 0.f;
             for (int jb = 0; jb < NJ; ++jb, ++bc) {
-                const int s = bc & 1, j0 = jb * 128;
+                if (int(bc % kTrGroups) != grp) continue;          // another warpgroup's block
+                const int j0 = jb * 128;
                 {
                     const int j = j0 + wt;
-                    ctl->jn[s][wt] = (j < S) ? inv_norm[sbase + j] * kTrLog2e : 0.f;
+                    jn_s[wt] = (j < S) ? inv_norm[sbase + j] * kTrLog2e : 0.f;
                     if (kPass == 2) {
                         const float zz = (j < S) ? z[sbase + j] : 1.f;
-                        ctl->jz[s][wt] = (zz > 0.f) ? 1.f / zz : 0.f;
+                        jz_s[wt] = (zz > 0.f) ? 1.f / zz : 0.f;
                     }
-                    named_bar_sync(1, 128);
+                    named_bar_sync(1 + grp, 128);
                 }
                 if (ok) {
-                    ok = tr_wait(ctl, &ctl->tfull[s], (bc >> 1) & 1u, status);
+                    ok = tr_wait(ctl, &ctl->tfull[grp], (bc / kTrGroups) & 1u, status);
                     ok = __all_sync(0xffffffffu, ok);
                 }
                 if (!ok) continue;                               // keeps the barrier pattern uniform
@@ -220,9 +228,9 @@ token_red_kernel(const __grid_constant__ CUtensorMap mapK, int n_slabs, int Hk, 
 #pragma unroll 1
                 for (int ch = 0; ch < 4; ++ch) {
                     float v[32];
-                    tmem_ld32(lane_addr + s * 128 + ch * 32, v);
-                    const float* jn = ctl->jn[s] + ch * 32;
-                    const float* jz = ctl->jz[s] + ch * 32;
+                    tmem_ld32(lane_addr + ch * 32, v);
+                    const float* jn = jn_s + ch * 32;
+                    const float* jz = jz_s + ch * 32;
                     if (interior) {
                         float e0 = 0.f, e1 = 0.f;
 #pragma unroll
@@ -249,9 +257,14 @@ token_red_kernel(const __grid_constant__ CUtensorMap mapK, int n_slabs, int Hk, 
                 }
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&ctl->tempty[s]);
+                if (lane == 0) mbar_arrive(&ctl->tempty[grp]);
             }
-            if (ok && i < S) {
+            // the warpgroups hold the sums over interleaved j blocks: the others hand their shares to the first
+            if (grp > 0) ctl->part[ic & 1][grp - 1][row] = accum;
+            named_bar_sync(1 + kTrGroups, 128 * kTrGroups);
+            if (grp == 0 && ok && i < S) {
+#pragma unroll
+                for (int g = 0; g < kTrGroups - 1; ++g) accum += ctl->part[ic & 1][g][row];
                 if (kPass == 1) z[sbase + i] = accum;
                 else tok_red[size_t(row0_of(slab)) + i] = accum / float(S);
             }
@@ -261,7 +274,7 @@ token_red_kernel(const __grid_constant__ CUtensorMap mapK, int n_slabs, int Hk, 
     __syncthreads();
     if (warp == 1) {
         tc_fence_after();
-        tmem_dealloc(tmem_base, 256);
+        tmem_dealloc(tmem_base, 128 * kTrGroups);
     }
 }
 
