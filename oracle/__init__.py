@@ -252,6 +252,29 @@ def token_redundancy(K_bits, eps=1e-6):
     return red
 
 
+# ------------------------------------------------------------------ per-token range append
+def append_token(sent_off, sent_id, new_sentence, gen_id):
+    """O15  Pre-eviction update of the cache-space range list for one appended token (Algorithm 1;
+    Section 4.1, "Updating Cache Ranges Before Eviction", Eq. "before" applied as soon as a token
+    arrives, i.e. with no tokens generated since: the range of the sentence the token belongs to ends
+    at the current cache length, and a new sentence begins right after the end of the previous one).
+    The cache stays fully partitioned: the trailing, still open sentence is the last range.
+
+    sent_off int32 [S+1] (CSR), sent_id int32 [S].  Returns the new (sent_off, sent_id)."""
+    off = [int(x) for x in sent_off]; ids = [int(x) for x in sent_id]
+    length = off[-1] if off else 0
+    ranges = [(off[i], off[i + 1] - 1) for i in range(len(ids))]              # inclusive (b, e)
+    if new_sentence or not ranges:
+        b = ranges[-1][1] + 1 if ranges else 0                                # b_i = e_{i-1} + 1
+        ranges.append((b, length))                                            # e_i = new length - 1
+        ids.append(int(gen_id))
+    else:
+        ranges[-1] = (ranges[-1][0], length)
+    new_off = [0] + [e + 1 for (_, e) in ranges]
+    assert all(ranges[i][0] == new_off[i] for i in range(len(ranges)))        # still a partition
+    return np.asarray(new_off, np.int32), np.asarray(ids, np.int32)
+
+
 # ------------------------------------------------------------------ batch drivers
 def score_batch(shape, K_bits, qwin_bits, kv_len, sent_off, n_sent, sigma, tau, eps, want_tok_imp=False):
     """shape: dict(batch,Hq,Hk,d,alpha,max_sent,slab_off,cap).  Returns dict of arrays."""

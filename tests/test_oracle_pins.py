@@ -630,6 +630,27 @@ def test_o14_closed_form_and_library():
     assert R3[3] > R[3] and R3[7] > np.median(R3)
 
 
+# ------------------------------------------------------------------ O15 range append
+def test_o15_append_token_hand_example():
+    off, ids = np.array([0, 3, 5], np.int32), np.array([7, 9], np.int32)
+    o1, i1 = oracle.append_token(off, ids, False, 11)                 # token 5 extends sentence 9
+    assert np.array_equal(o1, [0, 3, 6]) and np.array_equal(i1, [7, 9])
+    o2, i2 = oracle.append_token(o1, i1, True, 11)                    # token 6 starts sentence 11
+    assert np.array_equal(o2, [0, 3, 6, 7]) and np.array_equal(i2, [7, 9, 11])
+    o3, i3 = oracle.append_token(o2, i2, False, 12)
+    assert np.array_equal(o3, [0, 3, 6, 8]) and np.array_equal(i3, [7, 9, 11])
+    o0, i0 = oracle.append_token(np.array([0], np.int32), np.array([], np.int32), False, 4)   # empty cache
+    assert np.array_equal(o0, [0, 1]) and np.array_equal(i0, [4])
+    # a stream of tokens with delimiters reproduces the lengths of the sentences
+    lens = [4, 1, 6, 2]
+    off, ids = np.array([0], np.int32), np.array([], np.int32)
+    g = 0
+    for n, ln in enumerate(lens):
+        for t in range(ln):
+            off, ids = oracle.append_token(off, ids, t == 0, n)
+    assert np.array_equal(np.diff(off), lens) and np.array_equal(ids, [0, 1, 2, 3])
+
+
 def test_batch_drivers_match_slab_functions():
     cfg = W.config(0)
     L = W.make_layer(cfg)
