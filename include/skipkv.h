@@ -271,6 +271,23 @@ int skipkv_token_redundancy(const skipkv_shape* shape, const skipkv_params* para
                             const int32_t* kv_len, float* tok_red, void* ws, void* stream);
 
 /*
+ * skipkv_append_step -- the whole pre-eviction update of Algorithm 1 for one decode step (range append of
+ * Eq. "before" included), on the device.  Per (b, h): the new K/V row is written at kv_len and kv_len is
+ * incremented (as skipkv_append); the range list follows: when new_sent[b] != 0 (the previous token closed a
+ * sentence) or the slab has no sentence yet, a new sentence starts at this token with
+ * sent_id = gen_id[b]; the last sentence then ends at the newest token (sent_off[n_sent] = kv_len, entries
+ * above it mirror the length).  If q_win is non-null the step's query q[b][*] replaces slot `slot`
+ * (0 <= slot < window, host value, normally step % window) of the observation window q_win[b][*][slot].
+ * new_sent: device u8 [batch].  gen_id: device int32 [batch].  q: device bf16 [batch][Hq][128].
+ * A full slab (kv_len == cap) is left unchanged, a full range list (n_sent == max_sent) lets the token join
+ * the last sentence; both raise SKIPKV_STATUS_BAD_TABLE.
+ */
+int skipkv_append_step(const skipkv_shape* shape, void* K, void* V, const void* k_new, const void* v_new,
+                       int32_t* kv_len, int32_t* sent_off, int32_t* sent_id, int32_t* n_sent,
+                       const uint8_t* new_sent, const int32_t* gen_id, void* q_win, const void* q,
+                       int32_t slot, void* ws, void* stream);
+
+/*
  * skipkv_decode_attn_static -- skipkv_decode_attn for callers that cannot allocate device
  * memory and so have no workspace to pass.  (The paper has no counterpart: this is a packaging
  * variant of the same operation, not another step of the method.)  Typical callers: a serving

@@ -22,7 +22,8 @@ ERRORS = {-1: "SKIPKV_ERR_INVALID_ARG", -2: "SKIPKV_ERR_UNSUPPORTED", -3: "SKIPK
 SYMBOLS = ["skipkv_workspace_bytes", "skipkv_workspace_init", "skipkv_status", "skipkv_last_cuda_error",
            "skipkv_score", "skipkv_select", "skipkv_compact", "skipkv_decode_attn", "skipkv_steer",
            "skipkv_append", "skipkv_decode_attn_static", "skipkv_table_step", "skipkv_score_table",
-           "skipkv_select_fill", "skipkv_compact_fill", "skipkv_token_redundancy"]
+           "skipkv_select_fill", "skipkv_compact_fill", "skipkv_token_redundancy",
+           "skipkv_append_step"]
 
 
 class SkipKVError(RuntimeError):
@@ -202,6 +203,17 @@ def skipkv_token_redundancy(shape, params, K, kv_len, tok_red, ws, stream=None) 
     _check(lib().skipkv_token_redundancy(C.byref(shape), C.byref(params), _ptr(K, torch.bfloat16),
                                          _ptr(kv_len, torch.int32), _ptr(tok_red, torch.float32), _ptr(ws),
                                          _stream(stream)), "skipkv_token_redundancy")
+
+
+def skipkv_append_step(shape, K, V, k_new, v_new, kv_len, sent_off, sent_id, n_sent, new_sent, gen_id, q_win, q, slot,
+                       ws, stream=None) -> None:
+    _check(lib().skipkv_append_step(C.byref(shape), _ptr(K, torch.bfloat16), _ptr(V, torch.bfloat16),
+                                    _ptr(k_new, torch.bfloat16), _ptr(v_new, torch.bfloat16),
+                                    _ptr(kv_len, torch.int32), _ptr(sent_off, torch.int32),
+                                    _ptr(sent_id, torch.int32), _ptr(n_sent, torch.int32),
+                                    _ptr(new_sent, torch.uint8), _ptr(gen_id, torch.int32),
+                                    _ptr(q_win, torch.bfloat16), _ptr(q, torch.bfloat16), C.c_int32(slot), _ptr(ws),
+                                    _stream(stream)), "skipkv_append_step")
 
 
 def skipkv_decode_attn_static(shape, q, K, V, kv_len, out, hidden, steer_vec, alpha, flag, status=None,

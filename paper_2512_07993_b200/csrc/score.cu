@@ -587,14 +587,17 @@ score_pool_kernel(int Hk, int max_sent, int max_cap, const int32_t* cap, const i
 // persistent CTAs take the items round-robin, so barriers, tensor memory and descriptors are set up once and
 // the j-block ring keeps streaming from one item into the next.
 // ---------------------------------------------------------------------------------------
+constexpr int kGramGroups = 4;          // epilogue warpgroups = tensor-memory accumulators: one group's tensor-memory
+                                       // reads hide behind the arithmetic of the others
 struct GramCtl {
-    uint64_t afull, aempty, bfull[2], bempty[2], tfull[2], tempty[2];
+    uint64_t afull, aempty, bfull[2], bempty[2], tfull[kGramGroups], tempty[kGramGroups];
     uint32_t tmem_base;
     int abort_flag;
-    uint32_t wsum[8];
-    float invz[2][128];
+    uint32_t wsum[32];
+    alignas(16) float invz[kGramGroups][128];
+    float part[2][kGramGroups - 1][2][128];   // by item parity: the other groups' (sum, max) shares of a row
 };
-constexpr int kGramThreads = 6 * 32;
+constexpr int kGramThreads = (2 + 4 * kGramGroups) * 32;
 static size_t gram_smem_bytes(int slabs) { return 1024 + 6 * size_t(kOpBytes) + sizeof(GramCtl) + size_t(slabs + 1) * 4; }
 
 // Optional source of the sentence penalty: the lookup table T of one value per generation-space sentence,
@@ -643,6 +646,8 @@ score_gram_kernel(const __grid_constant__ CUtensorMap mapHi, const __grid_consta
         for (int s = 0; s < 2; ++s) {
             mbar_init(&ctl->bfull[s], 1);
             mbar_init(&ctl->bempty[s], 1);
+        }
+        for (int s = 0; s < kGramGroups; ++s) {
             mbar_init(&ctl->tfull[s], 1);
             mbar_init(&ctl->tempty[s], 4);
         }
@@ -651,7 +656,7 @@ score_gram_kernel(const __grid_constant__ CUtensorMap mapHi, const __grid_consta
         tmap_prefetch(&mapHi);
         tmap_prefetch(&mapLo);
     }
-    if (warp == 1) tmem_alloc(&ctl->tmem_base, 256);
+    if (warp == 1) tmem_alloc(&ctl->tmem_base, 128 * kGramGroups);
     {   // prefix of i blocks over slabs (block scan; every thread owns a contiguous block of slabs)
         const int per = (n_slabs + kGramThreads - 1) / kGramThreads;
         const int s0 = min(tid * per, n_slabs), s1 = min(s0 + per, n_slabs);
@@ -725,44 +730,48 @@ score_gram_kernel(const __grid_constant__ CUtensorMap mapHi, const __grid_consta
                 const int NJ = (sent_of(slab) + 127) >> 7;
                 ok = gram_wait(ctl, &ctl->afull, ic & 1u, status);
                 for (int jb = 0; jb < NJ && ok; ++jb, ++bc) {
-                    const int s = bc & 1;
+                    const int s = bc & 1, acc = bc % kGramGroups;
                     ok = gram_wait(ctl, &ctl->bfull[s], (bc >> 1) & 1u, status);
-                    if (ok && bc >= 2) ok = gram_wait(ctl, &ctl->tempty[s], ((bc >> 1) - 1) & 1u, status);
+                    if (ok && bc >= kGramGroups) ok = gram_wait(ctl, &ctl->tempty[acc], ((bc / kGramGroups) - 1) & 1u, status);
                     if (!ok) break;
                     tc_fence_after();
                     const uint32_t b_hi = smem_u32(Bt + size_t(s) * 2 * kOpBytes), b_lo = b_hi + kOpBytes;
-                    const uint32_t d = tmem_base + s * 128;
+                    const uint32_t d = tmem_base + acc * 128;
                     umma_tile_128x128x128(d, a_hi, b_hi, false);
                     umma_tile_128x128x128(d, a_hi, b_lo, true);
                     umma_tile_128x128x128(d, a_lo, b_hi, true);
-                    umma_commit(&ctl->tfull[s]);
+                    umma_commit(&ctl->tfull[acc]);
                     umma_commit(&ctl->bempty[s]);
                 }
                 if (ok) umma_commit(&ctl->aempty);                   // every MMA that reads this i block has completed
             }
         }
     } else {
-        const int quarter = warp & 3, wt = tid - 64;
-        const uint32_t lane_addr = tmem_base + (uint32_t(quarter * 32) << 16);
+        const int grp = (warp - 2) >> 2;                           // the accumulator this warpgroup drains
+        const int quarter = warp & 3, wt = (tid - 64) & 127;
+        const uint32_t lane_addr = tmem_base + (uint32_t(quarter * 32) << 16) + grp * 128;
+        float* invz_s = ctl->invz[grp];
         bool ok = true;
         int slab = 0;
-        uint32_t bc = 0;
-        for (int item = cta; item < n_items; item += G) {
+        uint32_t bc = 0, ic = 0;
+        for (int item = cta; item < n_items; item += G, ++ic) {
             while (ipref[slab + 1] <= item) ++slab;
             const int S = sent_of(slab), NJ = (S + 127) >> 7, rowbase = slab * max_sent;
             const int i0 = (item - ipref[slab]) * 128;
-            const int i = i0 + quarter * 32 + lane;
+            const int row = quarter * 32 + lane;
+            const int i = i0 + row;
             float accum = 0.f, mx = -INFINITY;
             for (int jb = 0; jb < NJ; ++jb, ++bc) {
-                const int s = bc & 1, j0 = jb * 128;
+                if (int(bc % kGramGroups) != grp) continue;        // another warpgroup's block
+                const int j0 = jb * 128;
                 if (kPass == 2) {
                     const int j = j0 + wt;
                     const float z = (j < S) ? sc_z[size_t(rowbase) + j] : 1.f;
-                    ctl->invz[s][wt] = (z > 0.f) ? 1.f / z : 0.f;
-                    named_bar_sync(1, 128);
+                    invz_s[wt] = (z > 0.f) ? 1.f / z : 0.f;
+                    named_bar_sync(1 + grp, 128);
                 }
                 if (ok) {
-                    ok = gram_wait(ctl, &ctl->tfull[s], (bc >> 1) & 1u, status);
+                    ok = gram_wait(ctl, &ctl->tfull[grp], (bc / kGramGroups) & 1u, status);
                     ok = __all_sync(0xffffffffu, ok);
                 }
                 if (!ok) continue;                               // keeps the barrier pattern uniform
@@ -771,8 +780,8 @@ score_gram_kernel(const __grid_constant__ CUtensorMap mapHi, const __grid_consta
 #pragma unroll 1
                 for (int ch = 0; ch < 4; ++ch) {
                     float v[32];
-                    tmem_ld32(lane_addr + s * 128 + ch * 32, v);
-                    const float* iz = ctl->invz[s] + ch * 32;
+                    tmem_ld32(lane_addr + ch * 32, v);
+                    const float* iz = invz_s + ch * 32;
                     if (interior) {
                         float e0 = 0.f, e1 = 0.f;
 #pragma unroll
@@ -808,9 +817,20 @@ score_gram_kernel(const __grid_constant__ CUtensorMap mapHi, const __grid_consta
                 }
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&ctl->tempty[s]);
+                if (lane == 0) mbar_arrive(&ctl->tempty[grp]);
             }
-            if (ok && i < S) {
+            // the warpgroups hold the sums (and maxima) over interleaved j blocks: the others hand theirs to the first
+            if (grp > 0) {
+                ctl->part[ic & 1][grp - 1][0][row] = accum;
+                if (kPass == 1) ctl->part[ic & 1][grp - 1][1][row] = mx;
+            }
+            named_bar_sync(1 + kGramGroups, 128 * kGramGroups);
+            if (grp == 0 && ok && i < S) {
+#pragma unroll
+                for (int g = 0; g < kGramGroups - 1; ++g) {
+                    accum += ctl->part[ic & 1][g][0][row];
+                    if (kPass == 1) mx = fmaxf(mx, ctl->part[ic & 1][g][1][row]);
+                }
                 const size_t o = size_t(rowbase) + i;
                 if (kPass == 1) {
                     sc_z[o] = accum;
@@ -832,7 +852,7 @@ score_gram_kernel(const __grid_constant__ CUtensorMap mapHi, const __grid_consta
     __syncthreads();
     if (warp == 1) {
         tc_fence_after();
-        tmem_dealloc(tmem_base, 256);
+        tmem_dealloc(tmem_base, 128 * kGramGroups);
     }
 }
 

@@ -1,0 +1,181 @@
+"""The decode loop of the method on the GPU, step by step against the CPU oracle (Algorithm 2 driven
+synthetically: random keys, values and queries stand in for the model; delimiters arrive at seeded sentence
+ends).  Every step appends a token (K/V row, range list, observation window), runs decode attention with the
+steering add on delimiter steps, and every `interval` steps evicts down to the budget.  The oracle mirrors the
+state on the host with its own functions.  After every step the attention output and the steered hidden state
+are compared; after every eviction the whole cache (rows, lengths, range tables) is compared bit for bit.  The
+eviction follows the usual contract: the GPU's keep flags equal the oracle's selection rule applied to the GPU's
+scores, the GPU's scores are within rtol 1e-3 of the oracle's, and the host state then follows those flags.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2512_07993_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+SIGMA, TAU, EPS = float(np.float32(0.1)), float(np.float32(0.95)), float(np.float32(1e-6))
+
+
+def close(name, got, ref, rtol=1e-3, atol=0.0):
+    got = np.asarray(got, np.float64); ref = np.asarray(ref, np.float64)
+    err = np.abs(got - ref) - (atol + rtol * np.abs(ref))
+    assert (err <= 0).all(), f"{name}: worst excess {err.max():.3e} at {int(err.argmax())}"
+
+
+@pytest.mark.parametrize("fill", [False, True])
+def test_decode_loop_with_periodic_eviction(fill):
+    from paper_2512_07993_b200 import build, binding as B
+    build.build()
+    steps, interval = 150, 32
+    cfg = W.config(0, cap_extra=48, budget=200, ctx_lo=300, ctx_hi=420, seed=91)
+    L = W.make_layer(cfg)
+    ms = int(L["max_sent"]) + steps                       # room for the sentences that will be appended
+    for key, fillv in (("sent_off", None), ("sent_id", -1)):
+        old = L[key]
+        new = np.zeros(old.shape[:2] + (ms + (1 if key == "sent_off" else 0),), np.int32)
+        new[..., :old.shape[2]] = old
+        new[..., old.shape[2]:] = old[..., -1:] if key == "sent_off" else -1
+        L[key] = new
+    L["max_sent"] = ms
+    D = B.DeviceLayer(L)
+    tok_keep = torch.zeros(D.K.shape[0], dtype=torch.uint8, device="cuda")
+    g, Hk, Hq, bt = cfg.group, cfg.n_kv_heads, cfg.n_q_heads, cfg.batch
+    r = np.random.Generator(np.random.Philox(2024))
+    # host mirror
+    Kh, Vh = W.bf16_bits(L["K"]).copy(), W.bf16_bits(L["V"]).copy()
+    kv = L["kv_len"].copy()
+    offs = {(b, h): L["sent_off"][b, h, :L["n_sent"][b, h] + 1].copy() for b in range(bt) for h in range(Hk)}
+    ids = {(b, h): L["sent_id"][b, h, :L["n_sent"][b, h]].copy() for b in range(bt) for h in range(Hk)}
+    qwin = W.bf16_bits(L["q_win"]).copy()
+    hidden = W.bf16_bits(L["hidden"]).copy()
+    steer_bits = W.bf16_bits(L["steer_vec"])
+    next_gen = np.array([int(L["n_sent"][b, 0]) for b in range(bt)], np.int32)
+    new_sent = np.zeros(bt, np.uint8)                      # the cached context ends inside an open sentence
+    left = r.integers(2, 12, size=bt)                      # tokens until each sequence's next delimiter
+    evictions = 0
+    for t in range(steps):
+        k_new = W.to_bf16(r.standard_normal((bt, Hk, 128), dtype=np.float32))
+        v_new = W.to_bf16(r.standard_normal((bt, Hk, 128), dtype=np.float32))
+        q = W.to_bf16(r.standard_normal((bt, Hq, 128), dtype=np.float32))
+        left -= 1
+        delim = (left == 0).astype(np.uint8)
+        left = np.where(left == 0, r.integers(2, 12, size=bt), left)
+        slot = t % cfg.window
+        gen_id = next_gen.copy()
+        # ---- GPU step
+        D.flag.copy_(torch.as_tensor(delim)); D.q.copy_(q)
+        B.skipkv_append_step(D.shape, D.K, D.V, k_new.cuda(), v_new.cuda(), D.kv_len, D.sent_off, D.sent_id, D.n_sent,
+                             torch.as_tensor(new_sent).cuda(), torch.as_tensor(gen_id).cuda(), D.q_win, D.q, slot, D.ws)
+        D.decode_attn(steer=True)
+        # ---- host mirror
+        kb, vb, qb = W.bf16_bits(k_new), W.bf16_bits(v_new), W.bf16_bits(q)
+        for b in range(bt):
+            for h in range(Hk):
+                row = W.slab_rows(L, b, h).start + int(kv[b, h])
+                Kh[row], Vh[row] = kb[b, h], vb[b, h]
+                offs[(b, h)], ids[(b, h)] = oracle.append_token(offs[(b, h)], ids[(b, h)], bool(new_sent[b]), gen_id[b])
+            kv[b, :] += 1
+            qwin[b, :, slot] = qb[b]
+        next_gen += new_sent
+        hidden = oracle.steer(hidden, steer_bits, L["alpha"], delim)
+        torch.cuda.synchronize()
+        assert D.status() == 0
+        assert np.array_equal(D.kv_len.cpu().numpy(), kv)
+        out = W.bf16_bits(D.out.cpu())
+        for b in range(bt):
+            for h in range(Hk):
+                rows = W.slab_rows(L, b, h)
+                n = int(kv[b, h])
+                _, o64 = oracle.decode_attn(qb[b, h * g:(h + 1) * g], Kh[rows][:n], Vh[rows][:n], n)
+                got = W.bits_to_bf16(out[b, h * g:(h + 1) * g]).float().numpy().astype(np.float64)
+                assert (np.abs(got - o64) / np.abs(o64).max(axis=-1, keepdims=True)).max() <= 2e-2, f"step {t} slab ({b},{h})"
+        assert np.array_equal(W.bf16_bits(D.hidden.cpu()), hidden), f"hidden at step {t}"
+        new_sent = delim.copy()                            # the token after a delimiter starts a sentence
+        if t % 37 == 5:                                    # range tables, now and then
+            so, sid, ns = D.sent_off.cpu().numpy(), D.sent_id.cpu().numpy(), D.n_sent.cpu().numpy()
+            for (b, h), off in offs.items():
+                S = len(ids[(b, h)])
+                assert ns[b, h] == S and np.array_equal(so[b, h, :S + 1], off) and (so[b, h, S + 1:] == off[-1]).all()
+                assert np.array_equal(sid[b, h, :S], ids[(b, h)])
+            assert np.array_equal(W.bf16_bits(D.q_win.cpu()), qwin)
+        # ---- eviction
+        if (t + 1) % interval == 0:
+            evictions += 1
+            D.score()
+            if fill:
+                B.skipkv_select_fill(D.shape, D.params, D.sent_score, D.tok_imp, D.sent_off, D.n_sent, D.keep, tok_keep,
+                                     D.kept_idx, D.n_kept, D.new_len, D.ws)
+            else:
+                D.select()
+            torch.cuda.synchronize()
+            sc, tok = D.sent_score.cpu().numpy(), D.tok_imp.cpu().numpy()
+            keep, tk = D.keep.cpu().numpy(), tok_keep.cpu().numpy()
+            if fill:
+                B.skipkv_compact_fill(D.shape, D.K, D.V, D.keep, tok_keep, D.sent_off, D.sent_id, D.n_sent, D.kv_len,
+                                      D.index_map, D.ws)
+            else:
+                D.compact()
+            torch.cuda.synchronize()
+            assert D.status() == 0
+            Kg, Vg = W.bf16_bits(D.K.cpu()), W.bf16_bits(D.V.cpu())
+            so, sid, ns, kvg = (x.cpu().numpy() for x in (D.sent_off, D.sent_id, D.n_sent, D.kv_len))
+            for b in range(bt):
+                for h in range(Hk):
+                    rows = W.slab_rows(L, b, h)
+                    n, off = int(kv[b, h]), offs[(b, h)]
+                    S = len(off) - 1
+                    o_tok = oracle.token_importance(Kh[rows][:n], qwin[b, h * g:(h + 1) * g])
+                    o_imp, vbar = oracle.pool(Kh[rows][:n], off, o_tok, EPS)
+                    _, o_red, o_lam = oracle.gram_terms(vbar, TAU)
+                    close(f"score step {t} ({b},{h})", sc[b, h, :S], oracle.final_score(o_imp, o_red, o_lam, SIGMA),
+                          rtol=1e-3, atol=1e-6)
+                    if fill:
+                        k_ref, t_ref, nl = oracle.select_fill(sc[b, h, :S], off, tok[rows][:n], cfg.budget, cfg.window)
+                        assert nl == min(n, cfg.budget)
+                    else:
+                        k_ref, _, nl = oracle.select(sc[b, h, :S], off, cfg.budget, cfg.window)
+                        t_ref = np.repeat(k_ref, np.diff(off))
+                    assert np.array_equal(keep[b, h, :S], k_ref), f"keep at step {t} ({b},{h})"
+                    Ko, Vo, _, nso, nsid = oracle.compact_tokens(Kh[rows][:n], Vh[rows][:n], t_ref, off, ids[(b, h)])
+                    m = Ko.shape[0]
+                    assert m == nl == int(kvg[b, h])
+                    assert np.array_equal(Kg[rows][:m], Ko) and np.array_equal(Vg[rows][:m], Vo)
+                    assert ns[b, h] == len(nsid) and np.array_equal(so[b, h, :len(nso)], nso)
+                    assert np.array_equal(sid[b, h, :len(nsid)], nsid)
+                    Kh[rows.start:rows.start + m] = Ko; Vh[rows.start:rows.start + m] = Vo
+                    kv[b, h] = m; offs[(b, h)] = nso; ids[(b, h)] = nsid
+    assert evictions == steps // interval and (kv <= cfg.budget + interval).all()
+
+
+def test_append_step_full_slab_and_full_range_list():
+    from paper_2512_07993_b200 import build, binding as B
+    build.build()
+    cfg = W.config(0, cap_extra=1)
+    L = W.make_layer(cfg)                                  # range tables exactly as long as the longest sequence needs
+    D = B.DeviceLayer(L)
+    bt, Hk = cfg.batch, cfg.n_kv_heads
+    z = torch.zeros(bt, Hk, 128, dtype=torch.bfloat16, device="cuda")
+    ones = torch.ones(bt, dtype=torch.uint8, device="cuda"); gen = torch.full((bt,), 999, dtype=torch.int32, device="cuda")
+    ns0, kv0 = D.n_sent.cpu().numpy().copy(), D.kv_len.cpu().numpy().copy()
+    so0 = D.sent_off.cpu().numpy().copy()
+    full = ns0 == D.max_sent                               # slabs whose range list has no free entry
+    assert full.any() and not full.all()
+    B.skipkv_append_step(D.shape, D.K, D.V, z, z, D.kv_len, D.sent_off, D.sent_id, D.n_sent, ones, gen, None, None, 0, D.ws)
+    torch.cuda.synchronize()
+    assert B.skipkv_status(D.ws, raise_on_error=False) == 0x4          # the full lists were reported
+    ns1, so1 = D.n_sent.cpu().numpy(), D.sent_off.cpu().numpy()
+    assert np.array_equal(D.kv_len.cpu().numpy(), kv0 + 1)
+    assert np.array_equal(ns1, np.where(full, ns0, ns0 + 1))           # full: the token joined the last sentence
+    for b in range(bt):
+        for h in range(Hk):
+            assert so1[b, h, ns1[b, h]] == kv0[b, h] + 1 and (so1[b, h, ns1[b, h]:] == kv0[b, h] + 1).all()
+            assert np.array_equal(so1[b, h, :ns0[b, h]], so0[b, h, :ns0[b, h]])
+    # the single spare row is used up: one more append leaves every slab unchanged and reports it
+    B.skipkv_append_step(D.shape, D.K, D.V, z, z, D.kv_len, D.sent_off, D.sent_id, D.n_sent, ones, gen, None, None, 0, D.ws)
+    torch.cuda.synchronize()
+    assert B.skipkv_status(D.ws, raise_on_error=False) == 0x4
+    assert np.array_equal(D.kv_len.cpu().numpy(), kv0 + 1) and np.array_equal(D.n_sent.cpu().numpy(), ns1)
+    B.skipkv_workspace_init(D.shape, D.ws)
