@@ -394,6 +394,32 @@ def test_append_then_decode(B):
     assert decode_err(W.bf16_bits(D.out.cpu()), o64) <= 2e-2
 
 
+@pytest.mark.parametrize("n,window", [(1, 32), (2, 32), (3, 20), (6, 32), (7, 9), (1, 128), (2, 100)])
+def test_every_group_size(B, n, window):
+    """Heads per KV head from 1 to 8 select different kernel instances: score and decode attention for the
+    sizes the named cases do not reach (1, 2, 3, 6, 7), with windows that fill one or several query blocks."""
+    cfg = W.config(0, name=f"group{n}", n_q_heads=2 * n, n_kv_heads=2, window=window, ctx_lo=300, ctx_hi=700,
+                   budget=200, seed=40 + n)
+    L = W.make_layer(cfg)
+    ref = oracle_scores(L)
+    D = B.DeviceLayer(L)
+    D.score(); D.decode_attn(steer=False)
+    torch.cuda.synchronize()
+    assert D.status() == 0
+    m = live_mask(L)
+    for name, got in (("imp", D.sent_imp), ("red", D.sent_red), ("lam", D.sent_lam)):
+        assert_close(name, got.cpu().numpy()[m], ref[name][m])
+    assert_close("score", D.sent_score.cpu().numpy()[m], ref["score"][m], rtol=1e-3, atol=1e-6)
+    tok = D.tok_imp.cpu().numpy()
+    for b in range(cfg.batch):
+        for h in range(cfg.n_kv_heads):
+            sl = W.slab_rows(L, b, h)
+            nl = int(L["kv_len"][b, h])
+            assert_close(f"tok_imp[{b},{h}]", tok[sl][:nl], ref["tok_imp"][sl][:nl])
+    _, o64 = oracle.decode_attn_batch(oshape(L), W.bf16_bits(L["q"]), W.bf16_bits(L["K"]), W.bf16_bits(L["V"]), L["kv_len"])
+    assert decode_err(W.bf16_bits(D.out.cpu()), o64) <= 2e-2
+
+
 def test_argument_errors(B):
     L = W.make_layer(W.config(0))
     D = B.DeviceLayer(L)
