@@ -27,10 +27,22 @@ def close(name, got, ref, rtol=1e-3, atol=0.0):
 
 @pytest.mark.parametrize("fill", [False, True])
 def test_decode_loop_with_periodic_eviction(fill):
+    """Small shape, every slab mirrored, every step checked."""
+    cfg = W.config(0, cap_extra=48, budget=200, ctx_lo=300, ctx_hi=420, seed=91)
+    run_loop(cfg, steps=150, interval=32, fill=fill, sampled=None, decode_every=1)
+
+
+def test_decode_loop_llama8b_shape_first_two_evictions():
+    """The decode-loop workload's shape (10 sequences, 8 KV heads x 4, 8192 cached tokens, budget 2048, eviction
+    every 128 steps, 32-query window ring, 256 spare rows per slab) through its first two evictions; three
+    slabs are mirrored by the oracle, decode attention is checked on them every 16th step and after each
+    eviction, invariants on every slab."""
+    run_loop(W.config(4), steps=260, interval=128, fill=False, sampled=[(0, 0), (4, 5), (9, 7)], decode_every=16)
+
+
+def run_loop(cfg, steps, interval, fill, sampled, decode_every):
     from paper_2512_07993_b200 import build, binding as B
     build.build()
-    steps, interval = 150, 32
-    cfg = W.config(0, cap_extra=48, budget=200, ctx_lo=300, ctx_hi=420, seed=91)
     L = W.make_layer(cfg)
     ms = int(L["max_sent"]) + steps                       # room for the sentences that will be appended
     for key, fillv in (("sent_off", None), ("sent_id", -1)):
@@ -43,18 +55,20 @@ def test_decode_loop_with_periodic_eviction(fill):
     D = B.DeviceLayer(L)
     tok_keep = torch.zeros(D.K.shape[0], dtype=torch.uint8, device="cuda")
     g, Hk, Hq, bt = cfg.group, cfg.n_kv_heads, cfg.n_q_heads, cfg.batch
+    slabs = sampled if sampled is not None else [(b, h) for b in range(bt) for h in range(Hk)]
     r = np.random.Generator(np.random.Philox(2024))
     # host mirror
     Kh, Vh = W.bf16_bits(L["K"]).copy(), W.bf16_bits(L["V"]).copy()
     kv = L["kv_len"].copy()
-    offs = {(b, h): L["sent_off"][b, h, :L["n_sent"][b, h] + 1].copy() for b in range(bt) for h in range(Hk)}
-    ids = {(b, h): L["sent_id"][b, h, :L["n_sent"][b, h]].copy() for b in range(bt) for h in range(Hk)}
+    offs = {(b, h): L["sent_off"][b, h, :L["n_sent"][b, h] + 1].copy() for (b, h) in slabs}
+    ids = {(b, h): L["sent_id"][b, h, :L["n_sent"][b, h]].copy() for (b, h) in slabs}
     qwin = W.bf16_bits(L["q_win"]).copy()
     hidden = W.bf16_bits(L["hidden"]).copy()
     steer_bits = W.bf16_bits(L["steer_vec"])
     next_gen = np.array([int(L["n_sent"][b, 0]) for b in range(bt)], np.int32)
     new_sent = np.zeros(bt, np.uint8)                      # the cached context ends inside an open sentence
-    left = r.integers(2, 12, size=bt)                      # tokens until each sequence's next delimiter
+    draw_len = lambda: r.integers(max(2, cfg.sent_lo // 2), cfg.sent_hi // 2 + 1, size=bt)
+    left = draw_len()                                      # tokens until each sequence's next delimiter
     evictions = 0
     for t in range(steps):
         k_new = W.to_bf16(r.standard_normal((bt, Hk, 128), dtype=np.float32))
@@ -62,7 +76,7 @@ def test_decode_loop_with_periodic_eviction(fill):
         q = W.to_bf16(r.standard_normal((bt, Hq, 128), dtype=np.float32))
         left -= 1
         delim = (left == 0).astype(np.uint8)
-        left = np.where(left == 0, r.integers(2, 12, size=bt), left)
+        left = np.where(left == 0, draw_len(), left)
         slot = t % cfg.window
         gen_id = next_gen.copy()
         # ---- GPU step
@@ -72,21 +86,20 @@ def test_decode_loop_with_periodic_eviction(fill):
         D.decode_attn(steer=True)
         # ---- host mirror
         kb, vb, qb = W.bf16_bits(k_new), W.bf16_bits(v_new), W.bf16_bits(q)
-        for b in range(bt):
-            for h in range(Hk):
-                row = W.slab_rows(L, b, h).start + int(kv[b, h])
-                Kh[row], Vh[row] = kb[b, h], vb[b, h]
-                offs[(b, h)], ids[(b, h)] = oracle.append_token(offs[(b, h)], ids[(b, h)], bool(new_sent[b]), gen_id[b])
-            kv[b, :] += 1
-            qwin[b, :, slot] = qb[b]
+        for (b, h) in slabs:
+            row = W.slab_rows(L, b, h).start + int(kv[b, h])
+            Kh[row], Vh[row] = kb[b, h], vb[b, h]
+            offs[(b, h)], ids[(b, h)] = oracle.append_token(offs[(b, h)], ids[(b, h)], bool(new_sent[b]), gen_id[b])
+        kv += 1
+        qwin[:, :, slot] = qb
         next_gen += new_sent
         hidden = oracle.steer(hidden, steer_bits, L["alpha"], delim)
         torch.cuda.synchronize()
         assert D.status() == 0
         assert np.array_equal(D.kv_len.cpu().numpy(), kv)
-        out = W.bf16_bits(D.out.cpu())
-        for b in range(bt):
-            for h in range(Hk):
+        if t % decode_every == 0 or t % interval == 0:      # the step after an eviction is always checked
+            out = W.bf16_bits(D.out.cpu())
+            for (b, h) in slabs:
                 rows = W.slab_rows(L, b, h)
                 n = int(kv[b, h])
                 _, o64 = oracle.decode_attn(qb[b, h * g:(h + 1) * g], Kh[rows][:n], Vh[rows][:n], n)
@@ -122,8 +135,14 @@ def test_decode_loop_with_periodic_eviction(fill):
             assert D.status() == 0
             Kg, Vg = W.bf16_bits(D.K.cpu()), W.bf16_bits(D.V.cpu())
             so, sid, ns, kvg = (x.cpu().numpy() for x in (D.sent_off, D.sent_id, D.n_sent, D.kv_len))
+            assert (kvg <= cfg.budget).all()
+            assert np.array_equal(D.new_len.cpu().numpy(), kvg)
             for b in range(bt):
                 for h in range(Hk):
+                    if (b, h) not in offs:
+                        assert kvg[b, h] <= cfg.budget and so[b, h, ns[b, h]] == kvg[b, h]
+                        kv[b, h] = kvg[b, h]
+                        continue
                     rows = W.slab_rows(L, b, h)
                     n, off = int(kv[b, h]), offs[(b, h)]
                     S = len(off) - 1

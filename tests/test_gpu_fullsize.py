@@ -45,6 +45,10 @@ def run_case(cfg, sample):
     D = B.DeviceLayer(L)
     D.score(); D.select(); D.compact(); D.decode_attn(steer=True)
     torch.cuda.synchronize()
+    check_layer(cfg, L, D, sample)
+
+
+def check_layer(cfg, L, D, sample):
     assert D.status() == 0
     g = cfg.group
     Kb, Vb, Qw, q = (W.bf16_bits(L[k]) for k in ("K", "V", "q_win", "q"))
@@ -110,6 +114,25 @@ def test_llama8b_32k_batch10_sampled_slabs():
     """The headline workload (batch 10, ragged 16K-32K tokens, budget 4096): three slabs recomputed."""
     cfg = W.config(2)
     run_case(cfg, [(0, 0), (4, 5), (9, 7)])
+
+
+def test_three_layers_back_to_back_on_one_stream():
+    """The 32-layer eviction pass in small: layers 0, 15 and 31 of the multi-layer workload (duplicate rate
+    10 %, 29 %, 50 %; sentence structure drawn per layer), each with its own cache and workspace, all twelve
+    calls enqueued on one stream with no synchronisation in between; one slab per layer recomputed."""
+    from paper_2512_07993_b200 import build, binding as B
+    build.build()
+    cfg = W.config(3, batch=4)
+    layers = (0, 15, 31)
+    Ls = [W.make_layer(cfg, layer=l, per_layer_sentences=True) for l in layers]
+    Ds = [B.DeviceLayer(L) for L in Ls]
+    for D in Ds:
+        D.score(); D.select(); D.compact(); D.decode_attn(steer=True)
+    torch.cuda.synchronize()
+    dup = [float((np.concatenate(L["dup_src"]) >= 0).mean()) for L in Ls]
+    assert dup[0] < dup[1] < dup[2]
+    for L, D, slab in zip(Ls, Ds, [(0, 3), (2, 0), (3, 7)]):
+        check_layer(cfg, L, D, [slab])
 
 
 def test_qwen14b_shape_sampled_slabs():
