@@ -273,6 +273,14 @@ decode_attn_kernel(int batch, int Hq, int Hk, int n_slabs, const int64_t* slab_o
         if (is_producer)
             for (int k = 0; k < kStages - 1; ++k) issue_next();
         DEC_TRACE(2);
+        // ------------------------------------------------------------------ steering add
+        // Independent of the attention (its own tensor), so it runs here, behind the wait for the first tiles
+        // whose copies were just issued, instead of lengthening the tail of the launch.
+        if (hidden != nullptr) {
+            const int vec_per_row = d_model / 8, total = batch * vec_per_row;
+            for (int i = cta * kDecThreads + tid; i < total; i += G * kDecThreads)
+                steer_vec8(i, vec_per_row, hidden, steer_vec, alpha, flag);
+        }
         bool first_tile = true;
 
         int slab = slab0, t = t_begin, c_stage = 0;
@@ -380,9 +388,9 @@ decode_attn_kernel(int batch, int Hq, int Hk, int n_slabs, const int64_t* slab_o
                 }
             }
             if (n_part > 1) {
-                __threadfence();
-                consumer_bar();
+                consumer_bar();                            // every thread's record stores are ordered before ...
                 if (tid == 0) {
+                    __threadfence();                       // ... this fence, which publishes them with the arrival below
                     const uint32_t old = atomicAdd(dec_cnt + slab, 1u);
                     const int last = (old == uint32_t(n_part - 1)) ? 1 : 0;
                     if (last) dec_cnt[slab] = 0u;          // self-resetting for the next launch
@@ -394,15 +402,29 @@ decode_attn_kernel(int batch, int Hq, int Hk, int n_slabs, const int64_t* slab_o
                     const float* r0 = dec_part + size_t(fc + slab) * n * kPartStride;
                     for (int idx = tid; idx < n * kHeadDim; idx += kConsWarps * 32) {
                         const int hl = idx / kHeadDim, c = idx % kHeadDim;
-                        float M = -INFINITY;
-                        for (int p = 0; p < n_part; ++p)
-                            M = fmaxf(M, __ldcg(r0 + (size_t(p) * n + hl) * kPartStride + 128));
-                        float L = 0.f, A = 0.f;
-                        for (int p = 0; p < n_part; ++p) {
-                            const float* rp = r0 + (size_t(p) * n + hl) * kPartStride;
-                            const float e = ex2(__ldcg(rp + 128) - M);
-                            L += __ldcg(rp + 129) * e;
-                            A += __ldcg(rp + c) * e;
+                        // four records per round: their loads are all in flight before the first is used
+                        float M = -INFINITY, L = 0.f, A = 0.f;
+                        for (int p0 = 0; p0 < n_part; p0 += 4) {
+                            float mm[4], ll[4], aa[4];
+#pragma unroll
+                            for (int k = 0; k < 4; ++k) {
+                                const float* rp = r0 + (size_t(min(p0 + k, n_part - 1)) * n + hl) * kPartStride;
+                                mm[k] = (p0 + k < n_part) ? __ldcg(rp + 128) : -INFINITY;
+                                ll[k] = __ldcg(rp + 129);
+                                aa[k] = __ldcg(rp + c);
+                            }
+                            float Mn = M;
+#pragma unroll
+                            for (int k = 0; k < 4; ++k) Mn = fmaxf(Mn, mm[k]);
+                            const float keep = ex2(M - Mn);              // first round: 2^(-inf) = 0
+                            L *= keep; A *= keep;
+#pragma unroll
+                            for (int k = 0; k < 4; ++k) {
+                                const float e = ex2(mm[k] - Mn);         // absent records: 2^(-inf) = 0
+                                L = fmaf(ll[k], e, L);
+                                A = fmaf(aa[k], e, A);
+                            }
+                            M = Mn;
                         }
                         o[idx] = __float2bfloat16_rn(L > 0.f ? A / L : 0.f);
                     }
@@ -421,12 +443,6 @@ decode_attn_kernel(int batch, int Hq, int Hk, int n_slabs, const int64_t* slab_o
             __nv_bfloat16* o = out + (size_t(b) * Hq + size_t(h) * n) * kHeadDim;
             for (int idx = tid; idx < n * kHeadDim; idx += kConsWarps * 32) o[idx] = __float2bfloat16_rn(0.f);
         }
-    }
-    // ---------------------------------------------------------------------- steering epilogue
-    if (hidden != nullptr) {
-        const int vec_per_row = d_model / 8, total = batch * vec_per_row;
-        for (int i = cta * kDecThreads + tid; i < total; i += G * kDecThreads)
-            steer_vec8(i, vec_per_row, hidden, steer_vec, alpha, flag);
     }
     DEC_TRACE(6);
 #ifdef SKIPKV_DEC_TRACE
