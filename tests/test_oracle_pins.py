@@ -682,3 +682,41 @@ def test_batch_drivers_match_slab_functions():
             assert np.array_equal(nso, cmp_["sent_off"][b, h, :len(nsid) + 1])
             o, _ = oracle.decode_attn(W.bf16_bits(L["q"][b, h * g:(h + 1) * g]), Ko, Vo, nl)
             assert np.array_equal(o, dec[b, h * g:(h + 1) * g])
+
+
+# ------------------------------------------------------------------ stored values
+def test_golden_oracle_outputs_unchanged():
+    """The oracle still produces the stored outputs for the seeded tiny slab (the file is written by
+    tests/golden/make_golden.py from the oracle alone)."""
+    import importlib.util, json, os
+    here = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden")
+    spec = importlib.util.spec_from_file_location("make_golden", os.path.join(here, "make_golden.py"))
+    mod = importlib.util.module_from_spec(spec); spec.loader.exec_module(mod)
+    now, stored = mod.compute(), json.load(open(os.path.join(here, "oracle_tiny_slab.json")))
+    assert now.keys() == stored.keys()
+    for k, v in stored.items():
+        if isinstance(v, list) and v and isinstance(v[0], float):
+            assert np.allclose(now[k], v, rtol=1e-10, atol=0.0), k
+        elif isinstance(v, float):
+            assert abs(now[k] - v) <= 1e-10 * abs(v), k
+        else:
+            assert now[k] == v, k
+
+
+def test_paper_hyperparameters_are_the_defaults():
+    """Values the paper prints (appendix, "Hyper-parameters") against the defaults of the binding and workloads."""
+    import os
+    from paper_2512_07993_b200 import binding
+    path = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", "paper_hyperparameters.txt")
+    hp = {}
+    for line in open(path):
+        if "=" in line and not line.startswith("#"):
+            k, v = line.split("=")
+            hp[k.strip()] = float(v)
+    p = binding.make_params()
+    assert abs(p.sigma - hp["sigma"]) < 1e-7 and hp["tau_low"] - 1e-7 <= p.tau <= hp["tau_high"]
+    cfg = W.config(4)
+    assert cfg.layers == 32 and hp["steer_layer_7b_8b"] < cfg.layers
+    L = W.make_layer(W.config(0))
+    k = (L["alpha"].astype(np.float64) - hp["alpha0_a"]) / hp["gamma"]           # alpha_t = alpha_0 + gamma * N_o
+    assert np.allclose(k, np.round(k), atol=1e-4) and (k >= 0).all()
