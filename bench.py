@@ -231,7 +231,18 @@ def time_extras(cfg, B, flush, clean, peaks, reps=10):
     out["compact_us"] = timed(D.compact, restore)
     restore(); select_fill()
     out["compact_fill_us"] = timed(compact_fill, restore)
+    # decode attention over the cache just compacted (exactly B rows per slab): contiguous slabs against the same
+    # number of rows behind a shuffled block table (page contents do not matter for the time)
+    slabs = cfg.batch * cfg.n_kv_heads
+    max_pages = (int(D.kv_len.max().item()) + 127) // 128
+    pool_pages = slabs * max_pages
+    Kp = torch.randn(pool_pages * 128, 128, device=dev).bfloat16(); Vp = torch.randn(pool_pages * 128, 128, device=dev).bfloat16()
+    table = torch.randperm(pool_pages, device=dev).to(torch.int32).reshape(cfg.batch, cfg.n_kv_heads, max_pages).contiguous()
+    out["decode_attn_us"] = timed(lambda: D.decode_attn(steer=True))
+    out["decode_attn_paged_us"] = timed(lambda: B.skipkv_decode_attn_paged(
+        D.shape, D.q, Kp, Vp, table, max_pages, D.kv_len, D.out, D.hidden, D.steer_vec, D.alpha, D.flag, D.ws))
     D.status()
+    del Kp, Vp
     del D, pristine, tok_keep
     torch.cuda.empty_cache()
     # token-level redundancy at the steady-state length of a budgeted cache: budget + 128 rows per slab

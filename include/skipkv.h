@@ -288,6 +288,21 @@ int skipkv_append_step(const skipkv_shape* shape, void* K, void* V, const void* 
                        int32_t slot, void* ws, void* stream);
 
 /*
+ * skipkv_decode_attn_paged -- skipkv_decode_attn over a paged cache, the layout of a paged-attention server
+ * (the paper's second host, appendix "System-Level Evaluation on vLLM").  K_pages and V_pages are pools of pages
+ * of SKIPKV_PAGE_ROWS rows of 128 bf16 (32 KB per page and tensor, page p at byte offset p * 32768, 16-byte
+ * aligned base); token t of slab (b, h) lives in row t % SKIPKV_PAGE_ROWS of page
+ * block_table[b][h][t / SKIPKV_PAGE_ROWS].  block_table: device int32 [batch][Hk][max_pages] (entries beyond the
+ * live pages are not read).  kv_len[b][h] <= min(cap[b], max_pages * SKIPKV_PAGE_ROWS); shape->slab_off is not
+ * used.  Everything else as skipkv_decode_attn; the two give bit-identical results for the same rows.
+ */
+#define SKIPKV_PAGE_ROWS 128
+int skipkv_decode_attn_paged(const skipkv_shape* shape, const void* q, const void* K_pages, const void* V_pages,
+                             const int32_t* block_table, int32_t max_pages, const int32_t* kv_len, void* out,
+                             void* hidden, const void* steer_vec, const float* alpha, const uint8_t* flag,
+                             void* ws, void* stream);
+
+/*
  * skipkv_decode_attn_static -- skipkv_decode_attn for callers that cannot allocate device
  * memory and so have no workspace to pass.  (The paper has no counterpart: this is a packaging
  * variant of the same operation, not another step of the method.)  Typical callers: a serving

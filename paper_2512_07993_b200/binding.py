@@ -23,7 +23,7 @@ SYMBOLS = ["skipkv_workspace_bytes", "skipkv_workspace_init", "skipkv_status", "
            "skipkv_score", "skipkv_select", "skipkv_compact", "skipkv_decode_attn", "skipkv_steer",
            "skipkv_append", "skipkv_decode_attn_static", "skipkv_table_step", "skipkv_score_table",
            "skipkv_select_fill", "skipkv_compact_fill", "skipkv_token_redundancy",
-           "skipkv_append_step"]
+           "skipkv_append_step", "skipkv_decode_attn_paged"]
 
 
 class SkipKVError(RuntimeError):
@@ -214,6 +214,16 @@ def skipkv_append_step(shape, K, V, k_new, v_new, kv_len, sent_off, sent_id, n_s
                                     _ptr(new_sent, torch.uint8), _ptr(gen_id, torch.int32),
                                     _ptr(q_win, torch.bfloat16), _ptr(q, torch.bfloat16), C.c_int32(slot), _ptr(ws),
                                     _stream(stream)), "skipkv_append_step")
+
+
+def skipkv_decode_attn_paged(shape, q, K_pages, V_pages, block_table, max_pages, kv_len, out, hidden, steer_vec, alpha,
+                             flag, ws, stream=None) -> None:
+    _check(lib().skipkv_decode_attn_paged(C.byref(shape), _ptr(q, torch.bfloat16), _ptr(K_pages, torch.bfloat16),
+                                          _ptr(V_pages, torch.bfloat16), _ptr(block_table, torch.int32),
+                                          C.c_int32(max_pages), _ptr(kv_len, torch.int32), _ptr(out, torch.bfloat16),
+                                          _ptr(hidden, torch.bfloat16), _ptr(steer_vec, torch.bfloat16),
+                                          _ptr(alpha, torch.float32), _ptr(flag, torch.uint8), _ptr(ws),
+                                          _stream(stream)), "skipkv_decode_attn_paged")
 
 
 def skipkv_decode_attn_static(shape, q, K, V, kv_len, out, hidden, steer_vec, alpha, flag, status=None,

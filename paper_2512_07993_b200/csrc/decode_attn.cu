@@ -159,7 +159,8 @@ __global__ void __launch_bounds__(kDecThreads, kCtasPerSm)
 decode_attn_kernel(int batch, int Hq, int Hk, int n_slabs, const int64_t* slab_off, const int32_t* cap,
                    const __nv_bfloat16* q, const uint8_t* K, const uint8_t* V, const int32_t* kv_len,
                    __nv_bfloat16* out, uint32_t* status, uint32_t* dec_cnt, float* dec_part, int d_model,
-                   __nv_bfloat16* hidden, const __nv_bfloat16* steer_vec, const float* alpha, const uint8_t* flag) {
+                   __nv_bfloat16* hidden, const __nv_bfloat16* steer_vec, const float* alpha, const uint8_t* flag,
+                   const int32_t* block_table, int max_pages) {
     extern __shared__ __align__(1024) uint8_t dsm[];
     uint8_t* ring = dsm;                                                     // kStages x (K tile, V tile)
     float* wpart = reinterpret_cast<float*>(dsm + kStages * 2 * kTileBytes);  // [8 warps][4 heads][132]
@@ -169,7 +170,11 @@ decode_attn_kernel(int batch, int Hq, int Hk, int n_slabs, const int64_t* slab_o
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     pdl_trigger();
     DEC_TRACE(0);
-    auto live = [&](int s) { return min(max(kv_len[s], 0), cap[s / Hk]); };   // live rows of slab s
+    // live rows of slab s; with a block table (paged cache) a slab cannot exceed its max_pages pages of kTileRows rows
+    auto live = [&](int s) {
+        const int c = block_table ? min(cap[s / Hk], max_pages * kTileRows) : cap[s / Hk];
+        return min(max(kv_len[s], 0), c);
+    };
     const int n = Hq / Hk;                     // heads per group
     const int NG = (n + 3) / 4;                // head groups of 4 (1 or 2)
     const int G = gridDim.x, cta = blockIdx.x;
@@ -234,7 +239,7 @@ decode_attn_kernel(int batch, int Hq, int Hk, int n_slabs, const int64_t* slab_o
         // ---- copy issue (thread 0 only): the CTA's k-th tile goes to stage k % kStages.  The cursor
         // walks the slab parts of this CTA's tile range; divisions and table reads happen once per part.
         const bool is_producer = (tid == 0);
-        int p_slab = slab0, p_t = t_begin, p_rows_left = 0, p_stage = 0;
+        int p_slab = slab0, p_t = t_begin, p_rows_left = 0, p_stage = 0, p_j = 0;
         uint32_t p_phase = 0;                           // parity of the previous use of p_stage (first lap: no wait)
         bool p_first_lap = true;
         const uint8_t *p_K = K, *p_V = V;
@@ -243,11 +248,19 @@ decode_attn_kernel(int batch, int Hq, int Hk, int n_slabs, const int64_t* slab_o
             if (p_rows_left <= 0) {
                 while (pref[p_slab + 1] <= p_t) ++p_slab;
                 const int j = p_t - pref[p_slab];
-                const size_t off =
-                    (slab_row0(slab_off, cap, Hk, p_slab / Hk, p_slab % Hk) + size_t(j) * kTileRows) * kRowBytes;
+                if (!block_table) {
+                    const size_t off =
+                        (slab_row0(slab_off, cap, Hk, p_slab / Hk, p_slab % Hk) + size_t(j) * kTileRows) * kRowBytes;
+                    p_K = K + off;
+                    p_V = V + off;
+                }
+                p_j = j;
+                p_rows_left = live(p_slab) - j * kTileRows;
+            }
+            if (block_table) {                          // paged cache: tile j of the slab is page block_table[slab][j]
+                const size_t off = size_t(max(block_table[size_t(p_slab) * max_pages + p_j], 0)) * kTileBytes;
                 p_K = K + off;
                 p_V = V + off;
-                p_rows_left = live(p_slab) - j * kTileRows;
             }
             if (!p_first_lap) {
                 if (sm->abort_flag || !mbar_wait(&sm->empty[p_stage], p_phase)) {
@@ -265,6 +278,7 @@ decode_attn_kernel(int batch, int Hq, int Hk, int n_slabs, const int64_t* slab_o
             p_V += kTileBytes;
             p_rows_left -= kTileRows;
             ++p_t;
+            ++p_j;
             if (++p_stage == kStages) {
                 p_stage = 0;
                 if (p_first_lap) p_first_lap = false; else p_phase ^= 1u;
@@ -464,9 +478,9 @@ extern "C" int skipkv_debug_set_trace(unsigned long long* p) {
 }
 #endif
 
-extern "C" int skipkv_decode_attn(const skipkv_shape* shape, const void* q, const void* K, const void* V,
-                                  const int32_t* kv_len, void* out, void* hidden, const void* steer_vec,
-                                  const float* alpha, const uint8_t* flag, void* ws, void* stream) {
+static int decode_impl(const skipkv_shape* shape, const void* q, const void* K, const void* V, const int32_t* kv_len,
+                       void* out, void* hidden, const void* steer_vec, const float* alpha, const uint8_t* flag,
+                       const int32_t* block_table, int max_pages, void* ws, void* stream) {
     if (int rc = check_shape(shape)) return rc;
     if (!q || !K || !V || !kv_len || !out) return SKIPKV_ERR_INVALID_ARG;
     if (hidden && (!steer_vec || !alpha || !flag || shape->d_model <= 0)) return SKIPKV_ERR_INVALID_ARG;
@@ -489,8 +503,24 @@ extern "C" int skipkv_decode_attn(const skipkv_shape* shape, const void* q, cons
         static_cast<const __nv_bfloat16*>(q), static_cast<const uint8_t*>(K), static_cast<const uint8_t*>(V), kv_len,
         static_cast<__nv_bfloat16*>(out), &reinterpret_cast<Header*>(w + L.header)->status,
         reinterpret_cast<uint32_t*>(w + L.dec_cnt), reinterpret_cast<float*>(w + L.dec_part), int(shape->d_model),
-        static_cast<__nv_bfloat16*>(hidden), static_cast<const __nv_bfloat16*>(steer_vec), alpha, flag));
+        static_cast<__nv_bfloat16*>(hidden), static_cast<const __nv_bfloat16*>(steer_vec), alpha, flag, block_table,
+        max_pages));
     return SKIPKV_OK;
+}
+
+extern "C" int skipkv_decode_attn(const skipkv_shape* shape, const void* q, const void* K, const void* V,
+                                  const int32_t* kv_len, void* out, void* hidden, const void* steer_vec,
+                                  const float* alpha, const uint8_t* flag, void* ws, void* stream) {
+    return decode_impl(shape, q, K, V, kv_len, out, hidden, steer_vec, alpha, flag, nullptr, 0, ws, stream);
+}
+
+extern "C" int skipkv_decode_attn_paged(const skipkv_shape* shape, const void* q, const void* K_pages,
+                                        const void* V_pages, const int32_t* block_table, int32_t max_pages,
+                                        const int32_t* kv_len, void* out, void* hidden, const void* steer_vec,
+                                        const float* alpha, const uint8_t* flag, void* ws, void* stream) {
+    if (!block_table || max_pages <= 0) return SKIPKV_ERR_INVALID_ARG;
+    return decode_impl(shape, q, K_pages, V_pages, kv_len, out, hidden, steer_vec, alpha, flag, block_table, max_pages, ws,
+                       stream);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -581,7 +611,7 @@ extern "C" int skipkv_decode_attn_static(const skipkv_shape* shape, const void* 
         static_cast<const __nv_bfloat16*>(q), static_cast<const uint8_t*>(K), static_cast<const uint8_t*>(V), kv_len,
         static_cast<__nv_bfloat16*>(out), status_word, reinterpret_cast<uint32_t*>(base + kStaticCntOff),
         reinterpret_cast<float*>(base + kStaticPartOff), shape->d_model, static_cast<__nv_bfloat16*>(hidden),
-        static_cast<const __nv_bfloat16*>(steer_vec), alpha, flag);
+        static_cast<const __nv_bfloat16*>(steer_vec), alpha, flag, static_cast<const int32_t*>(nullptr), 0);
     SKIPKV_CUDA(cudaGetLastError());
     return SKIPKV_OK;
 }
