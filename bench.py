@@ -245,6 +245,25 @@ def time_extras(cfg, B, flush, clean, peaks, reps=10):
     del Kp, Vp
     del D, pristine, tok_keep
     torch.cuda.empty_cache()
+    # one decode step of the decode-loop workload (cache a little above its budget of 2048): two launches against one
+    cfg4 = W.config(4, ctx_lo=2112, ctx_hi=2112, batch=cfg.batch)
+    D = B.DeviceLayer(W.make_layer(cfg4))
+    k_new = torch.randn(cfg4.batch, cfg4.n_kv_heads, 128, device=dev).bfloat16(); v_new = torch.randn_like(k_new)
+    zeros8 = torch.zeros(cfg4.batch, dtype=torch.uint8, device=dev); gen = torch.zeros(cfg4.batch, dtype=torch.int32, device=dev)
+    kv_in, kv_out = D.kv_len.clone(), torch.zeros_like(D.kv_len)
+    def two_launches():
+        D.kv_len.copy_(kv_in)
+        B.skipkv_append_step(D.shape, D.K, D.V, k_new, v_new, D.kv_len, D.sent_off, D.sent_id, D.n_sent, zeros8, gen, D.q_win,
+                             D.q, 0, D.ws)
+        D.decode_attn(steer=True)
+    def one_launch():
+        B.skipkv_decode_step(D.shape, D.q, k_new, v_new, D.K, D.V, kv_in, kv_out, D.sent_off, D.sent_id, D.n_sent, zeros8, gen,
+                             D.q_win, 0, D.out, D.hidden, D.steer_vec, D.alpha, D.flag, D.ws)
+    out["decode_step_two_launches_us"] = timed(two_launches)
+    out["decode_step_fused_us"] = timed(one_launch)
+    D.status()
+    del D
+    torch.cuda.empty_cache()
     # token-level redundancy at the steady-state length of a budgeted cache: budget + 128 rows per slab
     n_tok = cfg.budget + 128
     cfg_ss = W.config(0, batch=cfg.batch, n_q_heads=cfg.n_q_heads, n_kv_heads=cfg.n_kv_heads, window=cfg.window,

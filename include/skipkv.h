@@ -303,6 +303,22 @@ int skipkv_decode_attn_paged(const skipkv_shape* shape, const void* q, const voi
                              void* ws, void* stream);
 
 /*
+ * skipkv_decode_step -- one decode step of Algorithm 2 for one layer in a single launch: skipkv_append_step
+ * followed by skipkv_decode_attn (attention over the cache including the new row, steering add), fused.
+ * The new K/V row of (b, h) is written at kv_len_in[b][h] and attended to; the range list and the observation
+ * window are updated as by skipkv_append_step (q_win nullable: window untouched).  Lengths are read from
+ * kv_len_in and the new lengths written to kv_len_out, which must be a different buffer (the caller swaps the
+ * two between steps); sent_off, sent_id and n_sent are updated in place.  A slab without room is left
+ * unchanged (kv_len_out = kv_len_in, attention over the old rows) and raises SKIPKV_STATUS_BAD_TABLE, as does a
+ * full range list.  Contiguous slabs only.  Other arguments as skipkv_decode_attn.
+ */
+int skipkv_decode_step(const skipkv_shape* shape, const void* q, const void* k_new, const void* v_new, void* K,
+                       void* V, const int32_t* kv_len_in, int32_t* kv_len_out, int32_t* sent_off,
+                       int32_t* sent_id, int32_t* n_sent, const uint8_t* new_sent, const int32_t* gen_id,
+                       void* q_win, int32_t slot, void* out, void* hidden, const void* steer_vec,
+                       const float* alpha, const uint8_t* flag, void* ws, void* stream);
+
+/*
  * skipkv_decode_attn_static -- skipkv_decode_attn for callers that cannot allocate device
  * memory and so have no workspace to pass.  (The paper has no counterpart: this is a packaging
  * variant of the same operation, not another step of the method.)  Typical callers: a serving

@@ -23,7 +23,8 @@ SYMBOLS = ["skipkv_workspace_bytes", "skipkv_workspace_init", "skipkv_status", "
            "skipkv_score", "skipkv_select", "skipkv_compact", "skipkv_decode_attn", "skipkv_steer",
            "skipkv_append", "skipkv_decode_attn_static", "skipkv_table_step", "skipkv_score_table",
            "skipkv_select_fill", "skipkv_compact_fill", "skipkv_token_redundancy",
-           "skipkv_append_step", "skipkv_decode_attn_paged"]
+           "skipkv_append_step", "skipkv_decode_attn_paged",
+           "skipkv_decode_step"]
 
 
 class SkipKVError(RuntimeError):
@@ -224,6 +225,19 @@ def skipkv_decode_attn_paged(shape, q, K_pages, V_pages, block_table, max_pages,
                                           _ptr(hidden, torch.bfloat16), _ptr(steer_vec, torch.bfloat16),
                                           _ptr(alpha, torch.float32), _ptr(flag, torch.uint8), _ptr(ws),
                                           _stream(stream)), "skipkv_decode_attn_paged")
+
+
+def skipkv_decode_step(shape, q, k_new, v_new, K, V, kv_len_in, kv_len_out, sent_off, sent_id, n_sent, new_sent, gen_id,
+                       q_win, slot, out, hidden, steer_vec, alpha, flag, ws, stream=None) -> None:
+    _check(lib().skipkv_decode_step(C.byref(shape), _ptr(q, torch.bfloat16), _ptr(k_new, torch.bfloat16),
+                                    _ptr(v_new, torch.bfloat16), _ptr(K, torch.bfloat16), _ptr(V, torch.bfloat16),
+                                    _ptr(kv_len_in, torch.int32), _ptr(kv_len_out, torch.int32),
+                                    _ptr(sent_off, torch.int32), _ptr(sent_id, torch.int32),
+                                    _ptr(n_sent, torch.int32), _ptr(new_sent, torch.uint8),
+                                    _ptr(gen_id, torch.int32), _ptr(q_win, torch.bfloat16), C.c_int32(slot),
+                                    _ptr(out, torch.bfloat16), _ptr(hidden, torch.bfloat16),
+                                    _ptr(steer_vec, torch.bfloat16), _ptr(alpha, torch.float32),
+                                    _ptr(flag, torch.uint8), _ptr(ws), _stream(stream)), "skipkv_decode_step")
 
 
 def skipkv_decode_attn_static(shape, q, K, V, kv_len, out, hidden, steer_vec, alpha, flag, status=None,

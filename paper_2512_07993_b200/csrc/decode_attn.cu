@@ -56,12 +56,31 @@ __device__ __forceinline__ unsigned long long gtime() {
 #define DEC_TRACE(slot) do { } while (0)
 #endif
 
+// Optional fusion of the per-step bookkeeping into the decode launch (k_new == nullptr: plain decode attention).
+// The tile schedule covers the rows already cached; the CTA that owns a slab's last tile writes the new K/V row into
+// the cache, folds it into the attention as a one-row tile after the last streamed tile, and updates the slab's range
+// list and length when it flushes the segment.  A slab that was empty is handled with the zero-length slabs.  Lengths are read from kv_len and written to kv_len_out (a different buffer), so CTAs that
+// start late still derive the same tile schedule.
+struct StepArgs {
+    const uint4* k_new;          // [batch][Hk][16]
+    const uint4* v_new;
+    int32_t* kv_len_out;         // [batch][Hk]
+    int32_t* sent_off;           // range list, updated in place
+    int32_t* sent_id;
+    int32_t* n_sent;
+    const uint8_t* new_sent;     // [batch]
+    const int32_t* gen_id;       // [batch]
+    uint4* q_win;                // nullable: [batch][Hq][window][16]
+    int window, slot, max_sent;
+};
+
 struct DecSmem {
     uint64_t full[kStages];
     uint64_t empty[kStages];
     int abort_flag;
     int is_last;
     uint32_t wsum[kDecThreads / 32];
+    int step_n_sent, step_starts;          // fused step: range-list inputs of the slab whose tail this CTA holds
 };
 
 __device__ __forceinline__ void consumer_bar() { asm volatile("bar.sync 1, %0;" ::"n"(kConsWarps * 32) : "memory"); }
@@ -155,12 +174,15 @@ __device__ __forceinline__ void tile_rows(const uint8_t* Ks, const uint8_t* Vs, 
     }
 }
 
+// kStep: the launch also performs the per-step bookkeeping described at StepArgs (a separate instance, so that
+// plain decode attention carries none of it).
+template <bool kStep>
 __global__ void __launch_bounds__(kDecThreads, kCtasPerSm)
 decode_attn_kernel(int batch, int Hq, int Hk, int n_slabs, const int64_t* slab_off, const int32_t* cap,
                    const __nv_bfloat16* q, const uint8_t* K, const uint8_t* V, const int32_t* kv_len,
                    __nv_bfloat16* out, uint32_t* status, uint32_t* dec_cnt, float* dec_part, int d_model,
                    __nv_bfloat16* hidden, const __nv_bfloat16* steer_vec, const float* alpha, const uint8_t* flag,
-                   const int32_t* block_table, int max_pages) {
+                   const int32_t* block_table, int max_pages, StepArgs step) {
     extern __shared__ __align__(1024) uint8_t dsm[];
     uint8_t* ring = dsm;                                                     // kStages x (K tile, V tile)
     float* wpart = reinterpret_cast<float*>(dsm + kStages * 2 * kTileBytes);  // [8 warps][4 heads][132]
@@ -171,10 +193,10 @@ decode_attn_kernel(int batch, int Hq, int Hk, int n_slabs, const int64_t* slab_o
     pdl_trigger();
     DEC_TRACE(0);
     // live rows of slab s; with a block table (paged cache) a slab cannot exceed its max_pages pages of kTileRows rows
-    auto live = [&](int s) {
-        const int c = block_table ? min(cap[s / Hk], max_pages * kTileRows) : cap[s / Hk];
-        return min(max(kv_len[s], 0), c);
-    };
+    auto room = [&](int s) { return block_table ? min(cap[s / Hk], max_pages * kTileRows) : cap[s / Hk]; };
+    auto old_len = [&](int s) { return min(max(kv_len[s], 0), room(s)); };     // rows before this launch
+    // rows streamed through the tile ring; with the fused step the row being appended is folded in separately
+    auto live = [&](int s) { return old_len(s); };
     const int n = Hq / Hk;                     // heads per group
     const int NG = (n + 3) / 4;                // head groups of 4 (1 or 2)
     const int G = gridDim.x, cta = blockIdx.x;
@@ -184,6 +206,16 @@ decode_attn_kernel(int batch, int Hq, int Hk, int n_slabs, const int64_t* slab_o
         sm->abort_flag = 0;
         sm->is_last = 0;
         mbar_fence_init();
+    }
+    if (kStep) {
+        // the step's small inputs are read in the middle of the stream: start them towards L2 now (L2 is the point of
+        // coherence, so this is safe before the wait below)
+        const size_t row_bytes = size_t(n_slabs) * kRowBytes;
+        for (size_t o = size_t(cta * kDecThreads + tid) * 128; o < row_bytes; o += size_t(G) * kDecThreads * 128) {
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char*>(step.k_new) + o));
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char*>(step.v_new) + o));
+        }
+        if (tid * 32 < n_slabs) asm volatile("prefetch.global.L2 [%0];" ::"l"(step.n_sent + tid * 32));
     }
     pdl_wait();                                          // inputs (and the workspace) may come from the kernel before
     // tile prefix over slabs (block scan; every thread owns a contiguous block of slabs)
@@ -295,7 +327,36 @@ decode_attn_kernel(int batch, int Hq, int Hk, int n_slabs, const int64_t* slab_o
             for (int i = cta * kDecThreads + tid; i < total; i += G * kDecThreads)
                 steer_vec8(i, vec_per_row, hidden, steer_vec, alpha, flag);
         }
+        // fused step: this step's queries take their slot of the observation window
+        if (kStep && step.q_win != nullptr) {
+            const int total = batch * Hq * 16;
+            for (int i = cta * kDecThreads + tid; i < total; i += G * kDecThreads)
+                step.q_win[(size_t(i >> 4) * step.window + step.slot) * 16 + (i & 15)] = reinterpret_cast<const uint4*>(q)[i];
+        }
         bool first_tile = true;
+        // fused step: new length and range list of a slab after the append (all consumer threads call this together)
+        auto step_tables = [&](int slab_, int b_, bool appended, int S0, int starts_sentence) {
+            const int len = old_len(slab_);
+            const int new_len = appended ? len + 1 : len;
+            int32_t* so = step.sent_off + size_t(slab_) * (step.max_sent + 1);
+            const bool table_ok = S0 >= 0 && S0 <= step.max_sent;
+            int S = S0;
+            bool full_list = false;
+            if (appended && table_ok && (S0 == 0 || starts_sentence)) {
+                if (S0 < step.max_sent) S = S0 + 1; else full_list = true;   // full list: the token joins the last sentence
+            }
+            if (tid == 0) {
+                step.kv_len_out[slab_] = new_len;
+                if (appended && table_ok && S != S0) {
+                    if (S0 == 0) so[0] = 0;
+                    step.sent_id[size_t(slab_) * step.max_sent + S0] = step.gen_id[b_];
+                    step.n_sent[slab_] = S;
+                }
+                if (!appended || !table_ok || full_list) atomicOr(status, SKIPKV_STATUS_BAD_TABLE);
+            }
+            if (appended && table_ok)
+                for (int i = S + tid; i <= step.max_sent; i += kConsWarps * 32) so[i] = new_len;
+        };
 
         int slab = slab0, t = t_begin, c_stage = 0;
         uint32_t c_phase = 0;
@@ -305,6 +366,22 @@ decode_attn_kernel(int batch, int Hq, int Hk, int n_slabs, const int64_t* slab_o
             const int seg_end = min(t_end, pref[slab + 1]);
             const int b = slab / Hk, h = slab % Hk;
             int rows_left = live(slab) - (t - pref[slab]) * kTileRows;
+            const bool seg_append = kStep && old_len(slab) < room(slab);   // fused step: a row joins this slab
+            // fused step, this CTA holds the slab's last tile: fetch what the tail of the segment will need now, so
+            // that the loads are long complete when they are used
+            const bool own_tail = kStep && seg_end == pref[slab + 1];
+            if (own_tail) {
+                // the row being appended: into the cache, and staged as a one-row tile (K at byte 0, V at byte 2048 of
+                // the merge buffer, which is idle until the flush) for the fold-in after the last streamed tile
+                if (seg_append && warp == kConsWarps - 1) {
+                    const int part = lane >> 4, c = lane & 15;
+                    const uint4 val = (part ? step.v_new : step.k_new)[size_t(slab) * 16 + c];
+                    reinterpret_cast<uint4*>(reinterpret_cast<uint8_t*>(wpart) + part * 2048)[c] = val;
+                    const size_t row = slab_row0(slab_off, cap, Hk, b, h) + size_t(old_len(slab));
+                    reinterpret_cast<uint4*>(const_cast<uint8_t*>(part ? V : K))[row * 16 + c] = val;
+                }
+                if (tid == kDecThreads - 33) { sm->step_n_sent = step.n_sent[slab]; sm->step_starts = step.new_sent[b]; }
+            }
 #pragma unroll
             for (int hh = 0; hh < 4; ++hh) {
                 const int hl = hg * 4 + hh;
@@ -350,6 +427,18 @@ decode_attn_kernel(int batch, int Hq, int Hk, int n_slabs, const int64_t* slab_o
                 if (++c_stage == kStages) { c_stage = 0; c_phase ^= 1u; }
             }
 
+            // ---------------------------------------------------------- fused step: this CTA held the slab's last tile
+            if (own_tail && seg_append) {
+                consumer_bar();                            // the staged row is visible
+                if (warp < NG && !aborted)                 // one warp per head group folds the row into its running state
+                    tile_rows<true>(reinterpret_cast<const uint8_t*>(wpart), reinterpret_cast<const uint8_t*>(wpart) + 2048, 0, 1,
+                                    lane, q2, acc, m_run, l_run);
+                consumer_bar();                            // before the flush reuses the buffer
+            }
+            if (own_tail) {
+                consumer_bar();                            // the values parked at the start of the segment are visible
+                step_tables(slab, b, seg_append, sm->step_n_sent, sm->step_starts);
+            }
             // ---------------------------------------------------------- flush this (CTA, slab) segment
             if (t >= t_end) DEC_TRACE(4);
             // halves of the warp hold different rows: add them; finish the sum of p
@@ -455,7 +544,23 @@ decode_attn_kernel(int batch, int Hq, int Hk, int n_slabs, const int64_t* slab_o
             if (live(s) > 0) continue;
             const int b = s / Hk, h = s % Hk;
             __nv_bfloat16* o = out + (size_t(b) * Hq + size_t(h) * n) * kHeadDim;
-            for (int idx = tid; idx < n * kHeadDim; idx += kConsWarps * 32) o[idx] = __float2bfloat16_rn(0.f);
+            if (kStep && room(s) > 0) {
+                // fused step on an empty slab: the appended row is its only row, so every head's output is that value row
+                const __nv_bfloat16* vrow = reinterpret_cast<const __nv_bfloat16*>(step.v_new) + size_t(s) * kHeadDim;
+                for (int idx = tid; idx < n * kHeadDim; idx += kConsWarps * 32) o[idx] = vrow[idx % kHeadDim];
+                if (tid < 32) {
+                    const int part = tid >> 4, c = tid & 15;
+                    const size_t row = slab_row0(slab_off, cap, Hk, b, h);
+                    reinterpret_cast<uint4*>(const_cast<uint8_t*>(part ? V : K))[row * 16 + c] =
+                        (part ? step.v_new : step.k_new)[size_t(s) * 16 + c];
+                }
+                const int S0 = step.n_sent[s], starts = step.new_sent[b];
+                consumer_bar();                            // every thread has read n_sent before it changes
+                step_tables(s, b, true, S0, starts);
+            } else {
+                for (int idx = tid; idx < n * kHeadDim; idx += kConsWarps * 32) o[idx] = __float2bfloat16_rn(0.f);
+                if (kStep) step_tables(s, b, false, 0, 0);  // no room: unchanged, reported
+            }
         }
     }
     DEC_TRACE(6);
@@ -480,7 +585,7 @@ extern "C" int skipkv_debug_set_trace(unsigned long long* p) {
 
 static int decode_impl(const skipkv_shape* shape, const void* q, const void* K, const void* V, const int32_t* kv_len,
                        void* out, void* hidden, const void* steer_vec, const float* alpha, const uint8_t* flag,
-                       const int32_t* block_table, int max_pages, void* ws, void* stream) {
+                       const int32_t* block_table, int max_pages, const StepArgs& step, void* ws, void* stream) {
     if (int rc = check_shape(shape)) return rc;
     if (!q || !K || !V || !kv_len || !out) return SKIPKV_ERR_INVALID_ARG;
     if (hidden && (!steer_vec || !alpha || !flag || shape->d_model <= 0)) return SKIPKV_ERR_INVALID_ARG;
@@ -494,24 +599,25 @@ static int decode_impl(const skipkv_shape* shape, const void* q, const void* K, 
     const size_t smem = size_t(kStages) * 2 * kTileBytes + size_t(kConsWarps) * 4 * kWpStride * 4 + sizeof(DecSmem) +
                         size_t(L.slabs + 1) * 4;
     // set on every call: the attribute belongs to the current device's context, which a cached value would not track
-    SKIPKV_CUDA(cudaFuncSetAttribute(decode_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
+    auto kern = step.k_new ? decode_attn_kernel<true> : decode_attn_kernel<false>;
+    SKIPKV_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
     int grid = num_sms() * kCtasPerSm;
     if (grid > L.dec_max_ctas) grid = L.dec_max_ctas;
     SKIPKV_CUDA(launch_dependent(
-        decode_attn_kernel, dim3(grid), dim3(kDecThreads), smem, static_cast<cudaStream_t>(stream), int(shape->batch),
+        kern, dim3(grid), dim3(kDecThreads), smem, static_cast<cudaStream_t>(stream), int(shape->batch),
         int(shape->n_q_heads), int(shape->n_kv_heads), int(L.slabs), shape->slab_off, shape->cap,
         static_cast<const __nv_bfloat16*>(q), static_cast<const uint8_t*>(K), static_cast<const uint8_t*>(V), kv_len,
         static_cast<__nv_bfloat16*>(out), &reinterpret_cast<Header*>(w + L.header)->status,
         reinterpret_cast<uint32_t*>(w + L.dec_cnt), reinterpret_cast<float*>(w + L.dec_part), int(shape->d_model),
         static_cast<__nv_bfloat16*>(hidden), static_cast<const __nv_bfloat16*>(steer_vec), alpha, flag, block_table,
-        max_pages));
+        max_pages, step));
     return SKIPKV_OK;
 }
 
 extern "C" int skipkv_decode_attn(const skipkv_shape* shape, const void* q, const void* K, const void* V,
                                   const int32_t* kv_len, void* out, void* hidden, const void* steer_vec,
                                   const float* alpha, const uint8_t* flag, void* ws, void* stream) {
-    return decode_impl(shape, q, K, V, kv_len, out, hidden, steer_vec, alpha, flag, nullptr, 0, ws, stream);
+    return decode_impl(shape, q, K, V, kv_len, out, hidden, steer_vec, alpha, flag, nullptr, 0, StepArgs{}, ws, stream);
 }
 
 extern "C" int skipkv_decode_attn_paged(const skipkv_shape* shape, const void* q, const void* K_pages,
@@ -519,8 +625,29 @@ extern "C" int skipkv_decode_attn_paged(const skipkv_shape* shape, const void* q
                                         const int32_t* kv_len, void* out, void* hidden, const void* steer_vec,
                                         const float* alpha, const uint8_t* flag, void* ws, void* stream) {
     if (!block_table || max_pages <= 0) return SKIPKV_ERR_INVALID_ARG;
-    return decode_impl(shape, q, K_pages, V_pages, kv_len, out, hidden, steer_vec, alpha, flag, block_table, max_pages, ws,
-                       stream);
+    return decode_impl(shape, q, K_pages, V_pages, kv_len, out, hidden, steer_vec, alpha, flag, block_table, max_pages,
+                       StepArgs{}, ws, stream);
+}
+
+extern "C" int skipkv_decode_step(const skipkv_shape* shape, const void* q, const void* k_new, const void* v_new, void* K,
+                                  void* V, const int32_t* kv_len_in, int32_t* kv_len_out, int32_t* sent_off,
+                                  int32_t* sent_id, int32_t* n_sent, const uint8_t* new_sent, const int32_t* gen_id,
+                                  void* q_win, int32_t slot, void* out, void* hidden, const void* steer_vec,
+                                  const float* alpha, const uint8_t* flag, void* ws, void* stream) {
+    if (!k_new || !v_new || !kv_len_in || !kv_len_out || kv_len_in == kv_len_out || !sent_off || !sent_id || !n_sent ||
+        !new_sent || !gen_id)
+        return SKIPKV_ERR_INVALID_ARG;
+    if (int rc = check_shape(shape)) return rc;
+    if (shape->max_sent <= 0) return SKIPKV_ERR_INVALID_ARG;
+    if (q_win && (slot < 0 || slot >= shape->window)) return SKIPKV_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(k_new) | reinterpret_cast<uintptr_t>(v_new) | reinterpret_cast<uintptr_t>(q_win)) & 15)
+        return SKIPKV_ERR_INVALID_ARG;
+    StepArgs step{};
+    step.k_new = static_cast<const uint4*>(k_new); step.v_new = static_cast<const uint4*>(v_new);
+    step.kv_len_out = kv_len_out; step.sent_off = sent_off; step.sent_id = sent_id; step.n_sent = n_sent;
+    step.new_sent = new_sent; step.gen_id = gen_id; step.q_win = static_cast<uint4*>(q_win);
+    step.window = shape->window; step.slot = slot; step.max_sent = shape->max_sent;
+    return decode_impl(shape, q, K, V, kv_len_in, out, hidden, steer_vec, alpha, flag, nullptr, 0, step, ws, stream);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -598,7 +725,7 @@ extern "C" int skipkv_decode_attn_static(const skipkv_shape* shape, const void* 
                         size_t(slabs + 1) * 4;
     unsigned char* base = nullptr;
     if (int rc = static_setup(dev, &base)) return rc;
-    SKIPKV_CUDA(cudaFuncSetAttribute(decode_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
+    SKIPKV_CUDA(cudaFuncSetAttribute(decode_attn_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     // The array keeps whatever the previous call left: the status word and the arrival counters
     // must start at zero (the partial records are fully written before they are read).
@@ -606,12 +733,12 @@ extern "C" int skipkv_decode_attn_static(const skipkv_shape* shape, const void* 
     int grid = num_sms() * kCtasPerSm;
     if (grid > kStaticMaxCtas) grid = kStaticMaxCtas;
     uint32_t* status_word = status ? status : reinterpret_cast<uint32_t*>(base);
-    decode_attn_kernel<<<grid, kDecThreads, smem, st>>>(
+    decode_attn_kernel<false><<<grid, kDecThreads, smem, st>>>(
         shape->batch, shape->n_q_heads, shape->n_kv_heads, slabs, shape->slab_off, shape->cap,
         static_cast<const __nv_bfloat16*>(q), static_cast<const uint8_t*>(K), static_cast<const uint8_t*>(V), kv_len,
         static_cast<__nv_bfloat16*>(out), status_word, reinterpret_cast<uint32_t*>(base + kStaticCntOff),
         reinterpret_cast<float*>(base + kStaticPartOff), shape->d_model, static_cast<__nv_bfloat16*>(hidden),
-        static_cast<const __nv_bfloat16*>(steer_vec), alpha, flag, static_cast<const int32_t*>(nullptr), 0);
+        static_cast<const __nv_bfloat16*>(steer_vec), alpha, flag, static_cast<const int32_t*>(nullptr), 0, StepArgs{});
     SKIPKV_CUDA(cudaGetLastError());
     return SKIPKV_OK;
 }

@@ -25,11 +25,12 @@ def close(name, got, ref, rtol=1e-3, atol=0.0):
     assert (err <= 0).all(), f"{name}: worst excess {err.max():.3e} at {int(err.argmax())}"
 
 
-@pytest.mark.parametrize("fill", [False, True])
-def test_decode_loop_with_periodic_eviction(fill):
-    """Small shape, every slab mirrored, every step checked."""
+@pytest.mark.parametrize("fill,fused", [(False, False), (True, False), (False, True), (True, True)])
+def test_decode_loop_with_periodic_eviction(fill, fused):
+    """Small shape, every slab mirrored, every step checked; with the two launches per step (append_step, then
+    decode attention) and with the single fused launch (decode_step)."""
     cfg = W.config(0, cap_extra=48, budget=200, ctx_lo=300, ctx_hi=420, seed=91)
-    run_loop(cfg, steps=150, interval=32, fill=fill, sampled=None, decode_every=1)
+    run_loop(cfg, steps=150, interval=32, fill=fill, sampled=None, decode_every=1, fused=fused)
 
 
 def test_decode_loop_llama8b_shape_first_two_evictions():
@@ -40,7 +41,12 @@ def test_decode_loop_llama8b_shape_first_two_evictions():
     run_loop(W.config(4), steps=260, interval=128, fill=False, sampled=[(0, 0), (4, 5), (9, 7)], decode_every=16)
 
 
-def run_loop(cfg, steps, interval, fill, sampled, decode_every):
+def test_decode_loop_llama8b_shape_fused_step():
+    """The same workload shape with the fused step launch, through the first eviction."""
+    run_loop(W.config(4), steps=140, interval=128, fill=False, sampled=[(1, 2), (8, 0)], decode_every=16, fused=True)
+
+
+def run_loop(cfg, steps, interval, fill, sampled, decode_every, fused=False):
     from paper_2512_07993_b200 import build, binding as B
     build.build()
     L = W.make_layer(cfg)
@@ -54,6 +60,7 @@ def run_loop(cfg, steps, interval, fill, sampled, decode_every):
     L["max_sent"] = ms
     D = B.DeviceLayer(L)
     tok_keep = torch.zeros(D.K.shape[0], dtype=torch.uint8, device="cuda")
+    kv_len_other = torch.full_like(D.kv_len, -5)
     g, Hk, Hq, bt = cfg.group, cfg.n_kv_heads, cfg.n_q_heads, cfg.batch
     slabs = sampled if sampled is not None else [(b, h) for b in range(bt) for h in range(Hk)]
     r = np.random.Generator(np.random.Philox(2024))
@@ -81,9 +88,16 @@ def run_loop(cfg, steps, interval, fill, sampled, decode_every):
         gen_id = next_gen.copy()
         # ---- GPU step
         D.flag.copy_(torch.as_tensor(delim)); D.q.copy_(q)
-        B.skipkv_append_step(D.shape, D.K, D.V, k_new.cuda(), v_new.cuda(), D.kv_len, D.sent_off, D.sent_id, D.n_sent,
-                             torch.as_tensor(new_sent).cuda(), torch.as_tensor(gen_id).cuda(), D.q_win, D.q, slot, D.ws)
-        D.decode_attn(steer=True)
+        if fused:
+            B.skipkv_decode_step(D.shape, D.q, k_new.cuda(), v_new.cuda(), D.K, D.V, D.kv_len, kv_len_other, D.sent_off,
+                                 D.sent_id, D.n_sent, torch.as_tensor(new_sent).cuda(), torch.as_tensor(gen_id).cuda(),
+                                 D.q_win, slot, D.out, D.hidden, D.steer_vec, D.alpha, D.flag, D.ws)
+            D.kv_len, kv_len_other = kv_len_other, D.kv_len        # the new lengths are the current ones
+        else:
+            B.skipkv_append_step(D.shape, D.K, D.V, k_new.cuda(), v_new.cuda(), D.kv_len, D.sent_off, D.sent_id,
+                                 D.n_sent, torch.as_tensor(new_sent).cuda(), torch.as_tensor(gen_id).cuda(), D.q_win,
+                                 D.q, slot, D.ws)
+            D.decode_attn(steer=True)
         # ---- host mirror
         kb, vb, qb = W.bf16_bits(k_new), W.bf16_bits(v_new), W.bf16_bits(q)
         for (b, h) in slabs:
@@ -198,3 +212,89 @@ def test_append_step_full_slab_and_full_range_list():
     assert B.skipkv_status(D.ws, raise_on_error=False) == 0x4
     assert np.array_equal(D.kv_len.cpu().numpy(), kv0 + 1) and np.array_equal(D.n_sent.cpu().numpy(), ns1)
     B.skipkv_workspace_init(D.shape, D.ws)
+
+
+def test_decode_step_full_slab_and_full_range_list():
+    """The fused launch at its limits: a range list without a free entry lets the token join the last sentence;
+    a slab without a free row is attended over as it is; both are reported."""
+    from paper_2512_07993_b200 import build, binding as B
+    build.build()
+    cfg = W.config(0, cap_extra=1)
+    L = W.make_layer(cfg)
+    D = B.DeviceLayer(L)
+    bt, Hk = cfg.batch, cfg.n_kv_heads
+    g = torch.Generator().manual_seed(8)
+    k_new = torch.randn(bt, Hk, 128, generator=g).to(torch.bfloat16).cuda()
+    v_new = torch.randn(bt, Hk, 128, generator=g).to(torch.bfloat16).cuda()
+    ones = torch.ones(bt, dtype=torch.uint8, device="cuda"); gen = torch.full((bt,), 999, dtype=torch.int32, device="cuda")
+    ns0, kv0 = D.n_sent.cpu().numpy().copy(), D.kv_len.cpu().numpy().copy()
+    full = ns0 == D.max_sent
+    assert full.any() and not full.all()
+    kv_out = torch.full_like(D.kv_len, -3)
+
+    def step():
+        B.skipkv_decode_step(D.shape, D.q, k_new, v_new, D.K, D.V, D.kv_len, kv_out, D.sent_off, D.sent_id, D.n_sent, ones,
+                             gen, None, 0, D.out, None, None, None, None, D.ws)
+        torch.cuda.synchronize()
+
+    step()
+    assert B.skipkv_status(D.ws, raise_on_error=False) == 0x4
+    assert np.array_equal(kv_out.cpu().numpy(), kv0 + 1)
+    ns1, so1 = D.n_sent.cpu().numpy(), D.sent_off.cpu().numpy()
+    assert np.array_equal(ns1, np.where(full, ns0, ns0 + 1))
+    for b in range(bt):
+        for h in range(Hk):
+            assert (so1[b, h, ns1[b, h]:] == kv0[b, h] + 1).all()
+    out1 = D.out.clone()
+    # the same attention from the unfused entry point over the cache the step left behind
+    D.kv_len.copy_(kv_out)
+    D.decode_attn(steer=False)
+    torch.cuda.synchronize()
+    assert torch.equal(D.out.view(torch.int16), out1.view(torch.int16))
+    # no spare row left: the step changes nothing and attends over the rows that are there
+    kv_out.fill_(-3)
+    step()
+    assert B.skipkv_status(D.ws, raise_on_error=False) == 0x4
+    assert np.array_equal(kv_out.cpu().numpy(), kv0 + 1) and np.array_equal(D.n_sent.cpu().numpy(), ns1)
+    assert torch.equal(D.out.view(torch.int16), out1.view(torch.int16))
+    B.skipkv_workspace_init(D.shape, D.ws)
+
+
+def test_decode_step_on_an_empty_slab():
+    """A slab with no cached row: the appended row is its only row, so the attention output is that value row."""
+    from paper_2512_07993_b200 import build, binding as B
+    build.build()
+    cfg = W.config(0, cap_extra=4)
+    L = W.make_layer(cfg)
+    L["kv_len"][0, 1] = 0; L["n_sent"][0, 1] = 0; L["sent_off"][0, 1, :] = 0; L["sent_id"][0, 1, :] = -1
+    D = B.DeviceLayer(L)
+    bt, Hk, g = cfg.batch, cfg.n_kv_heads, cfg.group
+    gen_ = torch.Generator().manual_seed(9)
+    k_new = torch.randn(bt, Hk, 128, generator=gen_).to(torch.bfloat16); v_new = torch.randn(bt, Hk, 128, generator=gen_).to(torch.bfloat16)
+    zeros = torch.zeros(bt, dtype=torch.uint8, device="cuda"); gid = torch.full((bt,), 41, dtype=torch.int32, device="cuda")
+    kv_out = torch.full_like(D.kv_len, -3)
+    B.skipkv_decode_step(D.shape, D.q, k_new.cuda(), v_new.cuda(), D.K, D.V, D.kv_len, kv_out, D.sent_off, D.sent_id, D.n_sent,
+                         zeros, gid, None, 0, D.out, None, None, None, None, D.ws)
+    torch.cuda.synchronize()
+    assert D.status() == 0
+    assert np.array_equal(kv_out.cpu().numpy(), L["kv_len"] + 1)
+    out = D.out.cpu()
+    for q in range(g, 2 * g):                                        # the heads of KV head 1 of sequence 0
+        assert torch.equal(out[0, q].view(torch.int16), v_new[0, 1].view(torch.int16))
+    row = W.slab_rows(L, 0, 1).start
+    assert torch.equal(D.K[row].cpu().view(torch.int16), k_new[0, 1].view(torch.int16))
+    assert torch.equal(D.V[row].cpu().view(torch.int16), v_new[0, 1].view(torch.int16))
+    assert int(D.n_sent[0, 1]) == 1 and int(D.sent_id[0, 1, 0]) == 41
+    so = D.sent_off[0, 1].cpu().numpy()
+    assert so[0] == 0 and (so[1:] == 1).all()
+    # the other slabs: the same bits as the two-launch path on a fresh copy
+    D2 = B.DeviceLayer(L)
+    B.skipkv_append_step(D2.shape, D2.K, D2.V, k_new.cuda(), v_new.cuda(), D2.kv_len, D2.sent_off, D2.sent_id, D2.n_sent, zeros,
+                         gid, None, None, 0, D2.ws)
+    D2.decode_attn(steer=False)
+    torch.cuda.synchronize()
+    assert np.array_equal(D2.kv_len.cpu().numpy(), kv_out.cpu().numpy())
+    assert torch.equal(D2.sent_off, D.sent_off) and torch.equal(D2.n_sent, D.n_sent) and torch.equal(D2.sent_id, D.sent_id)
+    assert torch.equal(D2.K, D.K) and torch.equal(D2.V, D.V)
+    err = (D2.out.float() - D.out.float()).abs().max().item()
+    assert err <= 2e-2 * D2.out.float().abs().max().item()
