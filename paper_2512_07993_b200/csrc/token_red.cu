@@ -232,18 +232,18 @@ token_red_kernel(const __grid_constant__ CUtensorMap mapK, int n_slabs, int Hk, 
                     const float* jn = jn_s + ch * 32;
                     const float* jz = jz_s + ch * 32;
                     if (interior) {
-                        float e0 = 0.f, e1 = 0.f;
+                        // two elements per instruction (packed fp32 multiply / add): the epilogue is issue-bound
+                        float2 acc2 = make_float2(0.f, 0.f);
+                        const float2 inv2 = make_float2(inv_i, inv_i);
 #pragma unroll
                         for (int jj = 0; jj < 32; jj += 2) {
-                            if (kPass == 1) {
-                                e0 += tr_ex2(v[jj] * inv_i * jn[jj]);
-                                e1 += tr_ex2(v[jj + 1] * inv_i * jn[jj + 1]);
-                            } else {
-                                e0 = fmaf(tr_ex2(v[jj] * inv_i * jn[jj]), jz[jj], e0);
-                                e1 = fmaf(tr_ex2(v[jj + 1] * inv_i * jn[jj + 1]), jz[jj + 1], e1);
-                            }
+                            const float2 w = __fmul2_rn(__fmul2_rn(make_float2(v[jj], v[jj + 1]), inv2),
+                                                        *reinterpret_cast<const float2*>(jn + jj));
+                            const float2 e = make_float2(tr_ex2(w.x), tr_ex2(w.y));
+                            if (kPass == 1) acc2 = __fadd2_rn(acc2, e);
+                            else acc2 = __ffma2_rn(e, *reinterpret_cast<const float2*>(jz + jj), acc2);
                         }
-                        accum += e0 + e1;
+                        accum += acc2.x + acc2.y;
                     } else {
 #pragma unroll
                         for (int jj = 0; jj < 32; ++jj) {
