@@ -168,7 +168,6 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_consta
     const int G = gridDim.x, cta = blockIdx.x;
     const int n_slabs = a.n_slabs, Hk = a.Hk, RB = a.RB;
     pdl_trigger();
-    if (kSweep == 1) pdl_wait();                         // first kernel of the call: its inputs may come from the kernel before
     auto live = [&](int s) { return min(max(a.kv_len[s], 0), a.cap[s / Hk]); };
 
     if (tid == 0) {
@@ -188,6 +187,8 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_consta
         tmap_prefetch(&mapQ);
     }
     if (warp == 1) tmem_alloc(&ctl->tmem_base, 512);
+    // first kernel of the call: its inputs (lengths included) may come from the kernel before; the set-up above touched none
+    if (kSweep == 1) pdl_wait();
     // tile prefix over slabs (block scan; every thread owns a contiguous block of slabs)
     {
         const int per = (n_slabs + kThreads - 1) / kThreads;
