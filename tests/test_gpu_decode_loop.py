@@ -298,3 +298,53 @@ def test_decode_step_on_an_empty_slab():
     assert torch.equal(D2.K, D.K) and torch.equal(D2.V, D.V)
     err = (D2.out.float() - D.out.float()).abs().max().item()
     assert err <= 2e-2 * D2.out.float().abs().max().item()
+
+
+def test_fused_steps_back_to_back_without_synchronisation():
+    """Forty decode steps enqueued with no host synchronisation in between, once as two launches per step and once
+    as the fused launch (length buffers swapped every step): same cache, tables, lengths and last output."""
+    from paper_2512_07993_b200 import build, binding as B
+    build.build()
+    cfg = W.config(0, batch=3, cap_extra=64, ctx_lo=200, ctx_hi=500, seed=97)
+    L = W.make_layer(cfg)
+    ms = int(L["max_sent"]) + 48
+    for key in ("sent_off", "sent_id"):
+        old = L[key]
+        new = np.zeros(old.shape[:2] + (ms + (1 if key == "sent_off" else 0),), np.int32)
+        new[..., :old.shape[2]] = old
+        new[..., old.shape[2]:] = old[..., -1:] if key == "sent_off" else -1
+        L[key] = new
+    L["max_sent"] = ms
+    bt, Hk, Hq = cfg.batch, cfg.n_kv_heads, cfg.n_q_heads
+    g = torch.Generator().manual_seed(3)
+    steps = 40
+    ks = torch.randn(steps, bt, Hk, 128, generator=g).to(torch.bfloat16).cuda()
+    vs = torch.randn(steps, bt, Hk, 128, generator=g).to(torch.bfloat16).cuda()
+    qs = torch.randn(steps, bt, Hq, 128, generator=g).to(torch.bfloat16).cuda()
+    starts = (torch.rand(steps, bt, generator=g) < 0.2).to(torch.uint8).cuda()
+    flags = (torch.rand(steps, bt, generator=g) < 0.3).to(torch.uint8).cuda()
+    gids = (torch.arange(steps, dtype=torch.int32)[:, None] + 1000 * torch.arange(bt, dtype=torch.int32)[None, :]).cuda()
+
+    def run(fused):
+        D = B.DeviceLayer(L)
+        other = torch.zeros_like(D.kv_len)
+        for t in range(steps):
+            slot = t % cfg.window
+            if fused:
+                B.skipkv_decode_step(D.shape, qs[t], ks[t], vs[t], D.K, D.V, D.kv_len, other, D.sent_off, D.sent_id, D.n_sent,
+                                     starts[t], gids[t], D.q_win, slot, D.out, D.hidden, D.steer_vec, D.alpha, flags[t], D.ws)
+                D.kv_len, other = other, D.kv_len
+            else:
+                B.skipkv_append_step(D.shape, D.K, D.V, ks[t], vs[t], D.kv_len, D.sent_off, D.sent_id, D.n_sent, starts[t],
+                                     gids[t], D.q_win, qs[t], slot, D.ws)
+                B.skipkv_decode_attn(D.shape, qs[t], D.K, D.V, D.kv_len, D.out, D.hidden, D.steer_vec, D.alpha, flags[t], D.ws)
+        torch.cuda.synchronize()
+        assert D.status() == 0
+        return D
+
+    A, F = run(False), run(True)
+    assert torch.equal(A.kv_len, F.kv_len) and int(A.kv_len.min()) == int(L["kv_len"].min()) + steps
+    for name in ("K", "V", "sent_off", "sent_id", "n_sent", "q_win", "hidden"):
+        assert torch.equal(getattr(A, name), getattr(F, name)), name
+    err = (A.out.float() - F.out.float()).abs().max().item()
+    assert err <= 2e-2 * A.out.float().abs().max().item()
