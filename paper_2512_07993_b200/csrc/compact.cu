@@ -94,6 +94,7 @@ compact_plan_kernel(int Hk, int max_sent, const int64_t* slab_off, const int32_t
     __shared__ int wsum[kPlanThreads / 32][3];
     __shared__ int s_bad;
     __shared__ int s_npart, s_part[kMaxPartial][3], s_pos[64], s_wcnt[2];
+    __shared__ int s_next_begin[2];                      // old sent_off[base] of the next chunk of sentences (by chunk parity)
     // the move kernel is launched as a programmatic dependent: let its CTAs set themselves up while this grid runs
     pdl_trigger();
     pdl_wait();                                          // inputs may come from the kernel before
@@ -129,7 +130,11 @@ compact_plan_kernel(int Hk, int max_sent, const int64_t* slab_off, const int32_t
         const int i = base + tid;
         int b_i = 0, e_i = 0, id_i = -1, alive = 0, klen = 0;
         if (i < S) {
-            b_i = so[i]; e_i = so[i + 1]; id_i = sid[i];
+            // the table is rewritten in place, and the chunk before may already have overwritten so[base]: its
+            // last thread parked the old value
+            b_i = (tid == 0 && base > 0) ? s_next_begin[((base / kPlanThreads) & 1) ^ 1] : so[i];
+            e_i = so[i + 1]; id_i = sid[i];
+            if (tid == kPlanThreads - 1) s_next_begin[(base / kPlanThreads) & 1] = e_i;   // for thread 0 of the next chunk
             if (b_i < 0 || e_i < b_i || e_i > capb || (i == 0 && b_i != 0)) atomicOr(&s_bad, 1);
             else if (kp[i] != 0 && e_i > b_i) {
                 klen = e_i - b_i;

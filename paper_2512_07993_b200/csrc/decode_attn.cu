@@ -44,18 +44,6 @@ __device__ __forceinline__ float ex2(float x) {
     return y;
 }
 
-#ifdef SKIPKV_DEC_TRACE
-__device__ unsigned long long* g_dec_trace = nullptr;    // [ctas][8] nanosecond stamps (profiling builds only)
-__device__ __forceinline__ unsigned long long gtime() {
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-    return t;
-}
-#define DEC_TRACE(slot) do { if (g_dec_trace && threadIdx.x == 0) g_dec_trace[blockIdx.x * 8 + (slot)] = gtime(); } while (0)
-#else
-#define DEC_TRACE(slot) do { } while (0)
-#endif
-
 // Optional fusion of the per-step bookkeeping into the decode launch (k_new == nullptr: plain decode attention).
 // The tile schedule covers the rows already cached; the CTA that owns a slab's last tile writes the new K/V row into
 // the cache, folds it into the attention as a one-row tile after the last streamed tile, and updates the slab's range
@@ -191,7 +179,6 @@ decode_attn_kernel(int batch, int Hq, int Hk, int n_slabs, const int64_t* slab_o
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     pdl_trigger();
-    DEC_TRACE(0);
     // live rows of slab s; with a block table (paged cache) a slab cannot exceed its max_pages pages of kTileRows rows
     auto room = [&](int s) { return block_table ? min(cap[s / Hk], max_pages * kTileRows) : cap[s / Hk]; };
     auto old_len = [&](int s) { return min(max(kv_len[s], 0), room(s)); };     // rows before this launch
@@ -243,7 +230,6 @@ decode_attn_kernel(int batch, int Hq, int Hk, int n_slabs, const int64_t* slab_o
         if (tid == kDecThreads - 1) pref[n_slabs] = int(run);
         __syncthreads();
     }
-    DEC_TRACE(1);
     const int Ttot = pref[n_slabs];
     const int per_cta = max(1, (Ttot + G - 1) / G);
     const int t_begin = min(cta * per_cta, Ttot), t_end = min(t_begin + per_cta, Ttot);
@@ -318,7 +304,6 @@ decode_attn_kernel(int batch, int Hq, int Hk, int n_slabs, const int64_t* slab_o
         };
         if (is_producer)
             for (int k = 0; k < kStages - 1; ++k) issue_next();
-        DEC_TRACE(2);
         // ------------------------------------------------------------------ steering add
         // Independent of the attention (its own tensor), so it runs here, behind the wait for the first tiles
         // whose copies were just issued, instead of lengthening the tail of the launch.
@@ -333,7 +318,6 @@ decode_attn_kernel(int batch, int Hq, int Hk, int n_slabs, const int64_t* slab_o
             for (int i = cta * kDecThreads + tid; i < total; i += G * kDecThreads)
                 step.q_win[(size_t(i >> 4) * step.window + step.slot) * 16 + (i & 15)] = reinterpret_cast<const uint4*>(q)[i];
         }
-        bool first_tile = true;
         // fused step: new length and range list of a slab after the append (all consumer threads call this together)
         auto step_tables = [&](int slab_, int b_, bool appended, int S0, int starts_sentence) {
             const int len = old_len(slab_);
@@ -407,7 +391,6 @@ decode_attn_kernel(int batch, int Hq, int Hk, int n_slabs, const int64_t* slab_o
                         aborted = true;
                     }
                 }
-                if (first_tile) { DEC_TRACE(3); first_tile = false; }
                 if (!aborted) {
                     const uint8_t* Ks = ring + size_t(c_stage) * 2 * kTileBytes;
                     const uint8_t* Vs = Ks + kTileBytes;
@@ -440,7 +423,6 @@ decode_attn_kernel(int batch, int Hq, int Hk, int n_slabs, const int64_t* slab_o
                 step_tables(slab, b, seg_append, sm->step_n_sent, sm->step_starts);
             }
             // ---------------------------------------------------------- flush this (CTA, slab) segment
-            if (t >= t_end) DEC_TRACE(4);
             // halves of the warp hold different rows: add them; finish the sum of p
 #pragma unroll
             for (int hh = 0; hh < 4; ++hh)
@@ -535,7 +517,6 @@ decode_attn_kernel(int batch, int Hq, int Hk, int n_slabs, const int64_t* slab_o
             }
             consumer_bar();                                // wpart and is_last reusable
         }
-        DEC_TRACE(5);
         // after an abort copies may still be in flight: they must land before the CTA retires
         if (is_producer && sm->abort_flag)
             for (int st = 0; st < kStages; ++st) { mbar_wait(&sm->full[st], 0u, 1u << 16); mbar_wait(&sm->full[st], 1u, 1u << 16); }
@@ -563,25 +544,11 @@ decode_attn_kernel(int batch, int Hq, int Hk, int n_slabs, const int64_t* slab_o
             }
         }
     }
-    DEC_TRACE(6);
-#ifdef SKIPKV_DEC_TRACE
-    if (g_dec_trace && threadIdx.x == 0) {
-        unsigned smid;
-        asm volatile("mov.u32 %0, %smid;" : "=r"(smid));
-        g_dec_trace[blockIdx.x * 8 + 7] = smid;
-    }
-#endif
 }
 
 }  // namespace skipkv
 
 using namespace skipkv;
-
-#ifdef SKIPKV_DEC_TRACE
-extern "C" int skipkv_debug_set_trace(unsigned long long* p) {
-    return cudaMemcpyToSymbol(g_dec_trace, &p, sizeof(p)) == cudaSuccess ? 0 : -4;
-}
-#endif
 
 static int decode_impl(const skipkv_shape* shape, const void* q, const void* K, const void* V, const int32_t* kv_len,
                        void* out, void* hidden, const void* steer_vec, const float* alpha, const uint8_t* flag,

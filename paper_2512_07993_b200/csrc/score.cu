@@ -595,7 +595,8 @@ struct GramCtl {
     uint32_t tmem_base;
     int abort_flag;
     uint32_t wsum[32];
-    alignas(16) float invz[kGramGroups][128];
+    alignas(16) float invz[kGramGroups][2][128];   // by the parity of the group's block count: a warp that runs ahead
+                                                   // fills the other half while its siblings still read this one
     float part[2][kGramGroups - 1][2][128];   // by item parity: the other groups' (sum, max) shares of a row
 };
 constexpr int kGramThreads = (2 + 4 * kGramGroups) * 32;
@@ -658,6 +659,7 @@ score_gram_kernel(const __grid_constant__ CUtensorMap mapHi, const __grid_consta
         tmap_prefetch(&mapLo);
     }
     if (warp == 1) tmem_alloc(&ctl->tmem_base, 128 * kGramGroups);
+    pdl_wait();                                          // n_sent, the pooled keys and the row sums may come from the kernel before
     {   // prefix of i blocks over slabs (block scan; every thread owns a contiguous block of slabs)
         const int per = (n_slabs + kGramThreads - 1) / kGramThreads;
         const int s0 = min(tid * per, n_slabs), s1 = min(s0 + per, n_slabs);
@@ -683,7 +685,6 @@ score_gram_kernel(const __grid_constant__ CUtensorMap mapHi, const __grid_consta
         if (tid == kGramThreads - 1) ipref[n_slabs] = int(run);
         __syncthreads();
     }
-    pdl_wait();                                          // the pooled keys / row sums of the previous kernel
     const uint32_t tmem_base = ctl->tmem_base;
     const int n_items = ipref[n_slabs];
 
@@ -751,7 +752,6 @@ score_gram_kernel(const __grid_constant__ CUtensorMap mapHi, const __grid_consta
         const int grp = (warp - 2) >> 2;                           // the accumulator this warpgroup drains
         const int quarter = warp & 3, wt = (tid - 64) & 127;
         const uint32_t lane_addr = tmem_base + (uint32_t(quarter * 32) << 16) + grp * 128;
-        float* invz_s = ctl->invz[grp];
         bool ok = true;
         int slab = 0;
         uint32_t bc = 0, ic = 0;
@@ -765,6 +765,7 @@ score_gram_kernel(const __grid_constant__ CUtensorMap mapHi, const __grid_consta
             for (int jb = 0; jb < NJ; ++jb, ++bc) {
                 if (int(bc % kGramGroups) != grp) continue;        // another warpgroup's block
                 const int j0 = jb * 128;
+                float* invz_s = ctl->invz[grp][(bc / kGramGroups) & 1u];
                 if (kPass == 2) {
                     const int j = j0 + wt;
                     const float z = (j < S) ? sc_z[size_t(rowbase) + j] : 1.f;

@@ -30,8 +30,10 @@ struct TrCtl {
     uint32_t tmem_base;
     int abort_flag;
     uint32_t wsum[32];
-    alignas(16) float jn[kTrGroups][128];    // log2(e) / (|K_j| + eps) of the j block under an accumulator
-    alignas(16) float jz[kTrGroups][128];    // pass 2: 1 / Z_j
+    // per warpgroup, by the parity of its block count: a warp that runs ahead fills the other half while its
+    // siblings still read this one (the barrier of the block after orders the reuse)
+    alignas(16) float jn[kTrGroups][2][128]; // log2(e) / (|K_j| + eps) of the j block under an accumulator
+    alignas(16) float jz[kTrGroups][2][128]; // pass 2: 1 / Z_j
     float part[2][kTrGroups - 1][128];       // the other warpgroups' shares of an item's row sums (by item parity)
 };
 static size_t tr_smem_bytes(int slabs) { return 1024 + (1 + kTrStages) * size_t(kOpBytes) + sizeof(TrCtl) + size_t(slabs + 1) * 4; }
@@ -192,8 +194,6 @@ token_red_kernel(const __grid_constant__ CUtensorMap mapK, int n_slabs, int Hk, 
         const int grp = (warp - 2) >> 2;                           // the accumulator this warpgroup drains
         const int quarter = warp & 3, wt = (tid - 64) & 127;
         const uint32_t lane_addr = tmem_base + (uint32_t(quarter * 32) << 16) + grp * 128;
-        float* jn_s = ctl->jn[grp];
-        float* jz_s = ctl->jz[grp];
         bool ok = true;
         int slab = 0;
         uint32_t bc = 0, ic = 0;
@@ -209,6 +209,8 @@ token_red_kernel(const __grid_constant__ CUtensorMap mapK, int n_slabs, int Hk, 
             for (int jb = 0; jb < NJ; ++jb, ++bc) {
                 if (int(bc % kTrGroups) != grp) continue;          // another warpgroup's block
                 const int j0 = jb * 128;
+                float* jn_s = ctl->jn[grp][(bc / kTrGroups) & 1u];
+                float* jz_s = ctl->jz[grp][(bc / kTrGroups) & 1u];
                 {
                     const int j = j0 + wt;
                     jn_s[wt] = (j < S) ? inv_norm[sbase + j] * kTrLog2e : 0.f;

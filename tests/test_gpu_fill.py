@@ -184,6 +184,45 @@ def test_compact_fill_several_partial_sentences():
     check_compaction(L, D, cfg, keep, tk_ref)
 
 
+def test_compact_fill_partial_sentence_before_a_chunk_boundary_of_the_plan():
+    """More than 1024 sentences per slab (the plan walks the table 1024 sentences at a time and rewrites it in
+    place): every sentence up to and beyond the boundary survives and one of the first 1024 only in part, so the
+    rewritten offset at the boundary differs from the old one the next chunk needs."""
+    cfg = W.config(0, batch=1, ctx_lo=6200, ctx_hi=6400, sent_lo=3, sent_hi=6, budget=100000, seed=81)
+    L, D, B = device_layer(cfg)
+    r = np.random.Generator(np.random.Philox(321))
+    ms = int(L["max_sent"])
+    keep = np.zeros((cfg.batch, cfg.n_kv_heads, ms), np.uint8)
+    tk_dev = np.zeros(D.K.shape[0], np.uint8)
+    tk_ref = {}
+    for b in range(cfg.batch):
+        for h in range(cfg.n_kv_heads):
+            rows = W.slab_rows(L, b, h)
+            N, S = int(L["kv_len"][b, h]), int(L["n_sent"][b, h])
+            assert S > 1100
+            off = L["sent_off"][b, h, :S + 1]
+            k = np.ones(S, np.uint8)
+            k[1100 + h:] = (r.random(S - 1100 - h) < 0.5)
+            cut = [17, 1023][h % 2]                         # a partly kept sentence inside the first chunk
+            k[cut] = 2
+            t = np.zeros(N, np.uint8)
+            for i in range(S):
+                t[off[i]:off[i + 1]] = k[i]
+            t[off[cut]:off[cut + 1]] = 0
+            t[off[cut]] = 1                                 # one survivor
+            keep[b, h, :S] = k
+            tk_full = np.full(rows.stop - rows.start, 9, np.uint8)
+            tk_full[off[cut]:off[cut + 1]] = t[off[cut]:off[cut + 1]]
+            tk_dev[rows] = tk_full
+            tk_ref[(b, h)] = t
+    D.keep.copy_(torch.as_tensor(keep)); D.tok_keep.copy_(torch.as_tensor(tk_dev))
+    B.skipkv_compact_fill(D.shape, D.K, D.V, D.keep, D.tok_keep, D.sent_off, D.sent_id, D.n_sent, D.kv_len, D.index_map,
+                          D.ws)
+    torch.cuda.synchronize()
+    assert D.status() == 0
+    check_compaction(L, D, cfg, keep, tk_ref)
+
+
 def test_compact_fill_too_many_partial_sentences_is_reported():
     cfg = CASES["smoke"]()
     L, D, B = device_layer(cfg)
