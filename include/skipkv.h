@@ -94,6 +94,12 @@ int skipkv_workspace_bytes(const skipkv_shape* shape, size_t* bytes);
  * skipkv_status reported an error.  ws: device. */
 int skipkv_workspace_init(const skipkv_shape* shape, void* ws, void* stream);
 
+/* Set how many times a bounded device wait polls before it gives up and records SKIPKV_STATUS_*_TIMEOUT in the
+ * status word (every wait inside the kernels is bounded: a copy that never lands, or a hand-off another thread
+ * block never makes, ends the wait instead of hanging the GPU).  polls = 0 restores the default (about four million.  The value lives in the workspace and is kept by skipkv_workspace_init... until it is
+ * set again; it is read by the kernels enqueued after this call on `stream`.  ws: device. */
+int skipkv_set_wait_limit(void* ws, uint32_t polls, void* stream);
+
 /* Read and clear the device status word.  Synchronises `stream`.  *status_bits (host,
  * nullable) receives the SKIPKV_STATUS_* bits; returns SKIPKV_ERR_TIMEOUT if a wait ran out. */
 int skipkv_status(void* ws, void* stream, uint32_t* status_bits);

@@ -97,6 +97,8 @@ int check_shape(const skipkv_shape* s) {
     return SKIPKV_OK;
 }
 
+__global__ void ws_set_word_kernel(uint32_t* p, uint32_t v) { *p = v; }
+
 __global__ void ws_clear_kernel(uint32_t* p, size_t n_words) {
     for (size_t i = blockIdx.x * size_t(blockDim.x) + threadIdx.x; i < n_words; i += size_t(gridDim.x) * blockDim.x)
         p[i] = 0u;
@@ -128,7 +130,14 @@ int skipkv_workspace_init(const skipkv_shape* shape, void* ws, void* stream) {
     const WsLayout L = make_layout(*shape);
     // header + every counter region (everything before the decode partials)
     const size_t words = L.dec_part / 4;
-    ws_clear_kernel<<<64, 256, 0, static_cast<cudaStream_t>(stream)>>>(static_cast<uint32_t*>(ws), words);
+    ws_clear_kernel<<<592, 256, 0, static_cast<cudaStream_t>(stream)>>>(static_cast<uint32_t*>(ws), words);
+    SKIPKV_CUDA(cudaGetLastError());
+    return SKIPKV_OK;
+}
+
+int skipkv_set_wait_limit(void* ws, uint32_t polls, void* stream) {
+    if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255)) return SKIPKV_ERR_WORKSPACE;
+    ws_set_word_kernel<<<1, 1, 0, static_cast<cudaStream_t>(stream)>>>(&static_cast<Header*>(ws)->wait_limit, polls);
     SKIPKV_CUDA(cudaGetLastError());
     return SKIPKV_OK;
 }

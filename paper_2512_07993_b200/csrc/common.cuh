@@ -21,8 +21,10 @@ constexpr int kMaxQRows = 512;                // group * window
 struct Header {                // first 256 bytes of the workspace
     uint32_t status;           // SKIPKV_STATUS_* bits
     uint32_t compact_ticket;   // dynamic segment scheduler of the compaction kernel
-    uint32_t pad[62];
+    uint32_t wait_limit;       // polls a bounded device wait makes before it gives up; 0 = kDefaultWaitLimit
+    uint32_t pad[61];
 };
+constexpr uint32_t kDefaultWaitLimit = 1u << 22;
 
 struct WsLayout {
     size_t header;
@@ -195,6 +197,62 @@ __device__ __forceinline__ void bulk_wait_read_all() {
     asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
 }
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
+
+// The wait limit a workspace carries (skipkv_set_wait_limit); 0 stands for the default.
+__device__ __forceinline__ uint32_t load_wait_limit(const Header* hdr) {
+    const uint32_t v = *reinterpret_cast<const volatile uint32_t*>(&hdr->wait_limit);
+    return v ? v : kDefaultWaitLimit;
+}
+
+// Bounded wait of one role of a warp-specialised CTA: gives up after `limit` polls, or as soon as another role
+// of the CTA has flagged a failure; on expiry it flags the failure itself (status word + the CTA's abort flag).
+// The first probe is inline (the common case: the phase is already complete); the retry loop is kept out of line.
+static __device__ __noinline__ bool role_wait_slow(uint64_t* bar, uint32_t parity, uint32_t limit, int* abort_flag, uint32_t* status) {
+    if (*reinterpret_cast<volatile int*>(abort_flag)) return false;
+    for (uint32_t i = 0; i < limit; ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (i > 64) {
+            __nanosleep(64);
+            if ((i & 255) == 0 && *reinterpret_cast<volatile int*>(abort_flag)) return false;
+        }
+    }
+    atomicOr(status, SKIPKV_STATUS_COPY_TIMEOUT);
+    *reinterpret_cast<volatile int*>(abort_flag) = 1;
+    return false;
+}
+__device__ __forceinline__ bool role_wait(uint64_t* bar, uint32_t parity, uint32_t limit, int* abort_flag, uint32_t* status) {
+    if (mbar_try_wait(bar, parity)) return true;
+    return role_wait_slow(bar, parity, limit, abort_flag, status);
+}
+
+// Exclusive prefix of count(0..n-1) into pref[0..n] (pref[n] = total) by a whole CTA of kThreads threads; every thread
+// owns a contiguous block of indices.  wsum: kThreads / 32 words of shared memory.  Holds two CTA barriers; the
+// first one also publishes whatever the caller set up in shared memory before the call.
+template <int kThreads, typename F>
+__device__ __forceinline__ void cta_prefix(int n, F count, int* pref, uint32_t* wsum) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int per = (n + kThreads - 1) / kThreads;
+    const int s0 = min(tid * per, n), s1 = min(s0 + per, n);
+    uint32_t local = 0;
+    for (int s = s0; s < s1; ++s) local += uint32_t(count(s));
+    uint32_t inc = local;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const uint32_t x = __shfl_up_sync(0xffffffffu, inc, d);
+        if (lane >= d) inc += x;
+    }
+    if (lane == 31) wsum[warp] = inc;
+    __syncthreads();
+    uint32_t base = 0;
+    for (int w = 0; w < warp; ++w) base += wsum[w];
+    uint32_t run = base + inc - local;
+    for (int s = s0; s < s1; ++s) {
+        pref[s] = int(run);
+        run += uint32_t(count(s));
+    }
+    if (tid == kThreads - 1) pref[n] = int(run);
+    __syncthreads();
+}
 
 #endif  // __CUDACC__
 

@@ -254,6 +254,7 @@ compact_move_kernel(int n_slabs, int Hk, int max_sent, const int64_t* slab_off, 
     for (int w = 0; w < kMoveThreads / 32; ++w) max_nseg = max(max_nseg, s_red[w]);
     const uint32_t n_streams = 2u * n_slabs;
     const uint32_t n_tickets = n_streams * uint32_t(max_nseg);
+    const uint32_t limit = load_wait_limit(hdr);       // polls a wait makes before it gives up
     uint32_t phase = 0;
 
     for (;;) {
@@ -313,14 +314,14 @@ compact_move_kernel(int n_slabs, int Hk, int max_sent, const int64_t* slab_off, 
         }
         if (warp == 0) {
             // every lane observes the landing of the loads it is about to forward
-            int ok = mbar_wait(&bar, phase) ? 1 : 0;
+            int ok = mbar_wait(&bar, phase, limit) ? 1 : 0;
             if (lane == 0) {
                 if (!ok) atomicOr(&hdr->status, SKIPKV_STATUS_COPY_TIMEOUT);
                 // hand-off: wait until segments 0..j-1 of this stream are loaded, then publish j
                 volatile uint32_t* ld = cp_loaded + stream;
                 uint32_t spins = 0;
                 while (*ld < uint32_t(j)) {
-                    if (++spins > (1u << 22)) {
+                    if (++spins > limit) {
                         ok = 0;
                         atomicOr(&hdr->status, SKIPKV_STATUS_COMPACT_TIMEOUT);
                         break;

@@ -170,7 +170,7 @@ decode_attn_kernel(int batch, int Hq, int Hk, int n_slabs, const int64_t* slab_o
                    const __nv_bfloat16* q, const uint8_t* K, const uint8_t* V, const int32_t* kv_len,
                    __nv_bfloat16* out, uint32_t* status, uint32_t* dec_cnt, float* dec_part, int d_model,
                    __nv_bfloat16* hidden, const __nv_bfloat16* steer_vec, const float* alpha, const uint8_t* flag,
-                   const int32_t* block_table, int max_pages, StepArgs step) {
+                   const int32_t* block_table, int max_pages, StepArgs step, const uint32_t* wait_limit) {
     extern __shared__ __align__(1024) uint8_t dsm[];
     uint8_t* ring = dsm;                                                     // kStages x (K tile, V tile)
     float* wpart = reinterpret_cast<float*>(dsm + kStages * 2 * kTileBytes);  // [8 warps][4 heads][132]
@@ -205,6 +205,9 @@ decode_attn_kernel(int batch, int Hq, int Hk, int n_slabs, const int64_t* slab_o
         if (tid * 32 < n_slabs) asm volatile("prefetch.global.L2 [%0];" ::"l"(step.n_sent + tid * 32));
     }
     pdl_wait();                                          // inputs (and the workspace) may come from the kernel before
+    // polls a wait makes before it gives up: the workspace's setting, or the default without a workspace
+    uint32_t limit = kDefaultWaitLimit;
+    if (wait_limit) { const uint32_t v = *reinterpret_cast<const volatile uint32_t*>(wait_limit); if (v) limit = v; }
     // tile prefix over slabs (block scan; every thread owns a contiguous block of slabs)
     {
         const int per = (n_slabs + kDecThreads - 1) / kDecThreads;
@@ -281,7 +284,7 @@ decode_attn_kernel(int batch, int Hq, int Hk, int n_slabs, const int64_t* slab_o
                 p_V = V + off;
             }
             if (!p_first_lap) {
-                if (sm->abort_flag || !mbar_wait(&sm->empty[p_stage], p_phase)) {
+                if (sm->abort_flag || !mbar_wait(&sm->empty[p_stage], p_phase, limit)) {
                     if (!sm->abort_flag) atomicOr(status, SKIPKV_STATUS_COPY_TIMEOUT);
                     sm->abort_flag = 1;
                     return;
@@ -385,7 +388,7 @@ decode_attn_kernel(int batch, int Hq, int Hk, int n_slabs, const int64_t* slab_o
             for (; t < seg_end; ++t, rows_left -= kTileRows) {
                 if (is_producer) issue_next();                  // keeps kStages-1 tiles in flight
                 if (!aborted) {
-                    if (!mbar_wait(&sm->full[c_stage], c_phase) || sm->abort_flag) {
+                    if (!mbar_wait(&sm->full[c_stage], c_phase, limit) || sm->abort_flag) {
                         if (!sm->abort_flag) atomicOr(status, SKIPKV_STATUS_COPY_TIMEOUT);
                         sm->abort_flag = 1;
                         aborted = true;
@@ -577,7 +580,7 @@ static int decode_impl(const skipkv_shape* shape, const void* q, const void* K, 
         static_cast<__nv_bfloat16*>(out), &reinterpret_cast<Header*>(w + L.header)->status,
         reinterpret_cast<uint32_t*>(w + L.dec_cnt), reinterpret_cast<float*>(w + L.dec_part), int(shape->d_model),
         static_cast<__nv_bfloat16*>(hidden), static_cast<const __nv_bfloat16*>(steer_vec), alpha, flag, block_table,
-        max_pages, step));
+        max_pages, step, static_cast<const uint32_t*>(&reinterpret_cast<Header*>(w + L.header)->wait_limit)));
     return SKIPKV_OK;
 }
 
@@ -705,7 +708,8 @@ extern "C" int skipkv_decode_attn_static(const skipkv_shape* shape, const void* 
         static_cast<const __nv_bfloat16*>(q), static_cast<const uint8_t*>(K), static_cast<const uint8_t*>(V), kv_len,
         static_cast<__nv_bfloat16*>(out), status_word, reinterpret_cast<uint32_t*>(base + kStaticCntOff),
         reinterpret_cast<float*>(base + kStaticPartOff), shape->d_model, static_cast<__nv_bfloat16*>(hidden),
-        static_cast<const __nv_bfloat16*>(steer_vec), alpha, flag, static_cast<const int32_t*>(nullptr), 0, StepArgs{});
+        static_cast<const __nv_bfloat16*>(steer_vec), alpha, flag, static_cast<const int32_t*>(nullptr), 0, StepArgs{},
+        static_cast<const uint32_t*>(nullptr));
     SKIPKV_CUDA(cudaGetLastError());
     return SKIPKV_OK;
 }

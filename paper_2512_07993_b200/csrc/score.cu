@@ -55,7 +55,7 @@ struct SweepCtl {                       // barriers and small shared state, afte
     uint32_t tmem_base;
     int abort_flag;
     int landed;                         // sweep 2: tiles whose copy has completed (a monotone count for the pooling warps)
-    uint32_t wsum[16];
+    uint32_t wsum[32];
     alignas(16) float neg_lse[kSw2Groups][kMaxRB * 128];   // sweep 2: one copy per epilogue warpgroup (read as float4)
 };
 static_assert(offsetof(SweepCtl, neg_lse) % 16 == 0, "neg_lse is read with 16-byte loads");
@@ -73,22 +73,8 @@ struct SweepArgs {
     float* tok_imp_ws;
     float* vsum;                        // [slabs][max_sent][128] sums of key rows
     uint32_t* status;
+    const Header* hdr;
 };
-
-// Bounded wait that also gives up when another role of the CTA has flagged a failure.
-__device__ __forceinline__ bool ctl_wait(SweepCtl* ctl, uint64_t* bar, uint32_t parity, uint32_t* status) {
-    if (mbar_try_wait(bar, parity)) return true;
-    for (uint32_t i = 0; i < (1u << 22); ++i) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if (i > 64) {
-            __nanosleep(64);
-            if ((i & 255) == 0 && *reinterpret_cast<volatile int*>(&ctl->abort_flag)) return false;
-        }
-    }
-    atomicOr(status, SKIPKV_STATUS_COPY_TIMEOUT);
-    *reinterpret_cast<volatile int*>(&ctl->abort_flag) = 1;
-    return false;
-}
 
 // ---- sweep 1 epilogue: one accumulator (128 tokens) folded into the running (max, sum) of a row
 template <bool kMasked>
@@ -187,36 +173,13 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_consta
         tmap_prefetch(&mapQ);
     }
     if (warp == 1) tmem_alloc(&ctl->tmem_base, 512);
-    // first kernel of the call: its inputs (lengths included) may come from the kernel before; the set-up above touched none
-    if (kSweep == 1) pdl_wait();
-    // tile prefix over slabs (block scan; every thread owns a contiguous block of slabs)
-    {
-        const int per = (n_slabs + kThreads - 1) / kThreads;
-        const int s0 = min(tid * per, n_slabs), s1 = min(s0 + per, n_slabs);
-        uint32_t local = 0;
-        for (int s = s0; s < s1; ++s) local += uint32_t((live(s) + 127) >> 7);
-        uint32_t inc = local;
-#pragma unroll
-        for (int d = 1; d < 32; d <<= 1) {
-            const uint32_t x = __shfl_up_sync(0xffffffffu, inc, d);
-            if (lane >= d) inc += x;
-        }
-        if (lane == 31) ctl->wsum[warp] = inc;
-        tc_fence_before();
-        __syncthreads();                                 // also publishes barrier inits and the tmem address
-        tc_fence_after();
-        uint32_t base = 0;
-        for (int w = 0; w < warp; ++w) base += ctl->wsum[w];
-        uint32_t run = base + inc - local;
-        for (int s = s0; s < s1; ++s) {
-            pref[s] = int(run);
-            run += uint32_t((live(s) + 127) >> 7);
-        }
-        if (tid == kThreads - 1) pref[n_slabs] = int(run);
-        __syncthreads();
-    }
-    // (sweep 2) everything so far read only the call's inputs; what follows uses what sweep 1 wrote
+    // the lengths may come from the kernel before this call (and, in sweep 2, the records from sweep 1): the set-up
+    // above touched nothing that another kernel writes
     pdl_wait();
+    const uint32_t limit = load_wait_limit(a.hdr);
+    tc_fence_before();
+    cta_prefix<kThreads>(n_slabs, [&](int s) { return (live(s) + 127) >> 7; }, pref, ctl->wsum);   // also publishes the set-up
+    tc_fence_after();
     const uint32_t tmem_base = ctl->tmem_base;
     const int Ttot = pref[n_slabs];
     const int per_cta = max(1, (Ttot + G - 1) / G);
@@ -250,7 +213,7 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_consta
             for (int t = t_begin; t < t_end && ok; ++t) {
                 if (t == t_begin || pref[slab + 1] <= t) {
                     while (pref[slab + 1] <= t) ++slab;
-                    if (qlap > 0) ok = ctl_wait(ctl, &ctl->qempty, (qlap - 1) & 1u, a.status);
+                    if (qlap > 0) ok = role_wait(&ctl->qempty, (qlap - 1) & 1u, limit, &ctl->abort_flag, a.status);
                     if (!ok) break;
                     const int b = slab / Hk, h = slab % Hk;
                     mbar_expect_tx(&ctl->qfull, uint32_t(RB) * 2u * 128u * uint32_t(a.WB * n));
@@ -261,7 +224,7 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_consta
                     }
                     ++qlap;
                 }
-                if (lap > 0) ok = ctl_wait(ctl, &ctl->empty[stage], (lap - 1) & 1u, a.status);
+                if (lap > 0) ok = role_wait(&ctl->empty[stage], (lap - 1) & 1u, limit, &ctl->abort_flag, a.status);
                 if (!ok) break;
                 const long long row = (long long)slab_row0(a.slab_off, a.cap, Hk, slab / Hk, slab % Hk) +
                                       (long long)(t - pref[slab]) * 128;
@@ -288,11 +251,11 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_consta
             for (int t = t_begin; t < t_end && ok; ++t) {
                 if (t == t_begin || pref[slab + 1] <= t) {
                     while (pref[slab + 1] <= t) ++slab;
-                    ok = ctl_wait(ctl, &ctl->qfull, qlap & 1u, a.status);
+                    ok = role_wait(&ctl->qfull, qlap & 1u, limit, &ctl->abort_flag, a.status);
                     if (!ok) break;
                     ++qlap;
                 }
-                ok = ctl_wait(ctl, &ctl->full[stage], lap & 1u, a.status);
+                ok = role_wait(&ctl->full[stage], lap & 1u, limit, &ctl->abort_flag, a.status);
                 if (!ok) break;
                 if (kSweep == 2) {                       // pooling warps skip tiles, so they follow a count, not barrier phases
                     __threadfence_block();
@@ -301,7 +264,7 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_consta
                 const uint32_t k_smem = smem_u32(tiles + size_t(stage) * kOpBytes);
                 for (int k = 0; k < RB && ok; ++k, ++it) {
                     const int buf = it & (kAccBufs - 1), use = it / kAccBufs;
-                    if (use > 0) ok = ctl_wait(ctl, &ctl->tempty[buf], uint32_t(use - 1) & 1u, a.status);
+                    if (use > 0) ok = role_wait(&ctl->tempty[buf], uint32_t(use - 1) & 1u, limit, &ctl->abort_flag, a.status);
                     if (!ok) break;
                     tc_fence_after();
                     const uint32_t q_smem = smem_u32(qbuf + size_t(k) * kOpBytes);
@@ -341,7 +304,7 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_consta
                         if (k < RB && ok) {
                             const int it = tl * RB + k, buf = it & (kAccBufs - 1);
                             const int gj = (tl / kGroups) * RB + k;
-                            ok = ctl_wait(ctl, &ctl->tfull[g][gj & 3], uint32_t(gj >> 2) & 1u, a.status);
+                            ok = role_wait(&ctl->tfull[g][gj & 3], uint32_t(gj >> 2) & 1u, limit, &ctl->abort_flag, a.status);
                             ok = __all_sync(0xffffffffu, ok);
                             if (ok) {
                                 tc_fence_after();
@@ -396,7 +359,7 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_consta
                     if (k < RB && ok) {
                         const int it = tl * RB + k, buf = it & (kAccBufs - 1);
                         const int gj = (tl / kGroups) * RB + k;
-                        ok = ctl_wait(ctl, &ctl->tfull[g][gj & 3], uint32_t(gj >> 2) & 1u, a.status);
+                        ok = role_wait(&ctl->tfull[g][gj & 3], uint32_t(gj >> 2) & 1u, limit, &ctl->abort_flag, a.status);
                         ok = __all_sync(0xffffffffu, ok);
                         if (ok) {
                             tc_fence_after();
@@ -464,7 +427,7 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_consta
             if (ok) {                                           // wait (bounded) until the tile's copy has landed
                 uint32_t spins = 0;
                 while (*reinterpret_cast<volatile int*>(&ctl->landed) <= tl) {
-                    if (*reinterpret_cast<volatile int*>(&ctl->abort_flag) || ++spins > (1u << 22)) { ok = false; break; }
+                    if (*reinterpret_cast<volatile int*>(&ctl->abort_flag) || ++spins > limit) { ok = false; break; }
                     __nanosleep(64);
                 }
                 ok = __all_sync(0xffffffffu, ok);
@@ -612,25 +575,11 @@ struct LamTable {
     int Hk;
 };
 
-__device__ __forceinline__ bool gram_wait(GramCtl* ctl, uint64_t* bar, uint32_t parity, uint32_t* status) {
-    if (mbar_try_wait(bar, parity)) return true;
-    for (uint32_t i = 0; i < (1u << 22); ++i) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if (i > 64) {
-            __nanosleep(64);
-            if ((i & 255) == 0 && *reinterpret_cast<volatile int*>(&ctl->abort_flag)) return false;
-        }
-    }
-    atomicOr(status, SKIPKV_STATUS_COPY_TIMEOUT);
-    *reinterpret_cast<volatile int*>(&ctl->abort_flag) = 1;
-    return false;
-}
-
 template <int kPass>
 __global__ void __launch_bounds__(kGramThreads, 1)
 score_gram_kernel(const __grid_constant__ CUtensorMap mapHi, const __grid_constant__ CUtensorMap mapLo, int n_slabs,
                   int max_sent, const int32_t* n_sent, float sigma, float tau, float* sc_z, const float* sent_imp,
-                  float* sent_red, float* sent_lam, float* sent_score, LamTable ext, uint32_t* status) {
+                  float* sent_red, float* sent_lam, float* sent_score, LamTable ext, const Header* hdr) {
     extern __shared__ uint8_t gram_smem_raw[];
     const uint32_t raw = smem_u32(gram_smem_raw);
     uint8_t* At = gram_smem_raw + (((raw + 1023u) & ~1023u) - raw);              // hi, lo of the i block
@@ -660,31 +609,11 @@ score_gram_kernel(const __grid_constant__ CUtensorMap mapHi, const __grid_consta
     }
     if (warp == 1) tmem_alloc(&ctl->tmem_base, 128 * kGramGroups);
     pdl_wait();                                          // n_sent, the pooled keys and the row sums may come from the kernel before
-    {   // prefix of i blocks over slabs (block scan; every thread owns a contiguous block of slabs)
-        const int per = (n_slabs + kGramThreads - 1) / kGramThreads;
-        const int s0 = min(tid * per, n_slabs), s1 = min(s0 + per, n_slabs);
-        uint32_t local = 0;
-        for (int s = s0; s < s1; ++s) local += uint32_t((sent_of(s) + 127) >> 7);
-        uint32_t inc = local;
-#pragma unroll
-        for (int d = 1; d < 32; d <<= 1) {
-            const uint32_t x = __shfl_up_sync(0xffffffffu, inc, d);
-            if (lane >= d) inc += x;
-        }
-        if (lane == 31) ctl->wsum[warp] = inc;
-        tc_fence_before();
-        __syncthreads();                                 // also publishes barrier inits and the tmem address
-        tc_fence_after();
-        uint32_t base = 0;
-        for (int w = 0; w < warp; ++w) base += ctl->wsum[w];
-        uint32_t run = base + inc - local;
-        for (int s = s0; s < s1; ++s) {
-            ipref[s] = int(run);
-            run += uint32_t((sent_of(s) + 127) >> 7);
-        }
-        if (tid == kGramThreads - 1) ipref[n_slabs] = int(run);
-        __syncthreads();
-    }
+    uint32_t* status = const_cast<uint32_t*>(&hdr->status);
+    const uint32_t limit = load_wait_limit(hdr);
+    tc_fence_before();
+    cta_prefix<kGramThreads>(n_slabs, [&](int s) { return (sent_of(s) + 127) >> 7; }, ipref, ctl->wsum);   // i blocks per slab
+    tc_fence_after();
     const uint32_t tmem_base = ctl->tmem_base;
     const int n_items = ipref[n_slabs];
 
@@ -697,7 +626,7 @@ score_gram_kernel(const __grid_constant__ CUtensorMap mapHi, const __grid_consta
                 while (ipref[slab + 1] <= item) ++slab;
                 const int S = sent_of(slab), NJ = (S + 127) >> 7, rowbase = slab * max_sent;
                 const int i0 = (item - ipref[slab]) * 128;
-                if (ic > 0) ok = gram_wait(ctl, &ctl->aempty, (ic - 1) & 1u, status);
+                if (ic > 0) ok = role_wait(&ctl->aempty, (ic - 1) & 1u, limit, &ctl->abort_flag, status);
                 if (!ok) break;
                 mbar_expect_tx(&ctl->afull, 2 * kOpBytes);
                 tma_load_2d(At, &mapHi, 0, rowbase + i0, &ctl->afull);
@@ -706,7 +635,7 @@ score_gram_kernel(const __grid_constant__ CUtensorMap mapHi, const __grid_consta
                 tma_load_2d(At + kOpBytes + kOpHalfBytes, &mapLo, 64, rowbase + i0, &ctl->afull);
                 for (int jb = 0; jb < NJ && ok; ++jb, ++bc) {
                     const int s = bc & 1;
-                    if (bc >= 2) ok = gram_wait(ctl, &ctl->bempty[s], ((bc >> 1) - 1) & 1u, status);
+                    if (bc >= 2) ok = role_wait(&ctl->bempty[s], ((bc >> 1) - 1) & 1u, limit, &ctl->abort_flag, status);
                     if (!ok) break;
                     uint8_t* dst = Bt + size_t(s) * 2 * kOpBytes;
                     mbar_expect_tx(&ctl->bfull[s], 2 * kOpBytes);
@@ -730,11 +659,11 @@ score_gram_kernel(const __grid_constant__ CUtensorMap mapHi, const __grid_consta
             for (int item = cta; item < n_items && ok; item += G, ++ic) {
                 while (ipref[slab + 1] <= item) ++slab;
                 const int NJ = (sent_of(slab) + 127) >> 7;
-                ok = gram_wait(ctl, &ctl->afull, ic & 1u, status);
+                ok = role_wait(&ctl->afull, ic & 1u, limit, &ctl->abort_flag, status);
                 for (int jb = 0; jb < NJ && ok; ++jb, ++bc) {
                     const int s = bc & 1, acc = bc % kGramGroups;
-                    ok = gram_wait(ctl, &ctl->bfull[s], (bc >> 1) & 1u, status);
-                    if (ok && bc >= kGramGroups) ok = gram_wait(ctl, &ctl->tempty[acc], ((bc / kGramGroups) - 1) & 1u, status);
+                    ok = role_wait(&ctl->bfull[s], (bc >> 1) & 1u, limit, &ctl->abort_flag, status);
+                    if (ok && bc >= kGramGroups) ok = role_wait(&ctl->tempty[acc], ((bc / kGramGroups) - 1) & 1u, limit, &ctl->abort_flag, status);
                     if (!ok) break;
                     tc_fence_after();
                     const uint32_t b_hi = smem_u32(Bt + size_t(s) * 2 * kOpBytes), b_lo = b_hi + kOpBytes;
@@ -773,7 +702,7 @@ score_gram_kernel(const __grid_constant__ CUtensorMap mapHi, const __grid_consta
                     named_bar_sync(1 + grp, 128);
                 }
                 if (ok) {
-                    ok = gram_wait(ctl, &ctl->tfull[grp], (bc / kGramGroups) & 1u, status);
+                    ok = role_wait(&ctl->tfull[grp], (bc / kGramGroups) & 1u, limit, &ctl->abort_flag, status);
                     ok = __all_sync(0xffffffffu, ok);
                 }
                 if (!ok) continue;                               // keeps the barrier pattern uniform
@@ -906,6 +835,7 @@ static int score_impl(const skipkv_shape* shape, const skipkv_params* params, co
     a.slab_off = shape->slab_off; a.cap = shape->cap; a.kv_len = kv_len; a.sent_off = sent_off; a.n_sent = n_sent;
     a.sc_part = reinterpret_cast<float2*>(w + L.sc_part);
     a.tok_imp_user = tok_imp; a.tok_imp_ws = sc_tok; a.vsum = vsum; a.status = status;
+    a.hdr = reinterpret_cast<const Header*>(w + L.header);
     const size_t max_smem = 227 * 1024;
     const size_t fixed1 = 1024 + size_t(a.RB) * kOpBytes + sizeof(SweepCtl) + size_t(L.slabs + 1) * 4;
     if (fixed1 + kOpBytes > max_smem) return SKIPKV_ERR_UNSUPPORTED;
@@ -953,10 +883,10 @@ static int score_impl(const skipkv_shape* shape, const skipkv_params* params, co
         SKIPKV_CUDA(cudaFuncSetAttribute(score_gram_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(gsmem)));
         SKIPKV_CUDA(launch_dependent(score_gram_kernel<1>, dim3(ggrid), dim3(kGramThreads), gsmem, st, mapHi, mapLo, L.slabs,
                                      shape->max_sent, n_sent, params->sigma, params->tau, sc_z, sent_imp, sent_red, sent_lam,
-                                     sent_score, ext, status));
+                                     sent_score, ext, reinterpret_cast<const Header*>(w + L.header)));
         SKIPKV_CUDA(launch_dependent(score_gram_kernel<2>, dim3(ggrid), dim3(kGramThreads), gsmem, st, mapHi, mapLo, L.slabs,
                                      shape->max_sent, n_sent, params->sigma, params->tau, sc_z, sent_imp, sent_red, sent_lam,
-                                     sent_score, ext, status));
+                                     sent_score, ext, reinterpret_cast<const Header*>(w + L.header)));
     }
     return SKIPKV_OK;
 }

@@ -68,25 +68,11 @@ token_norm_kernel(int Hk, int max_cap, const int64_t* slab_off, const int32_t* c
     }
 }
 
-__device__ __forceinline__ bool tr_wait(TrCtl* ctl, uint64_t* bar, uint32_t parity, uint32_t* status) {
-    if (mbar_try_wait(bar, parity)) return true;
-    for (uint32_t i = 0; i < (1u << 22); ++i) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if (i > 64) {
-            __nanosleep(64);
-            if ((i & 255) == 0 && *reinterpret_cast<volatile int*>(&ctl->abort_flag)) return false;
-        }
-    }
-    atomicOr(status, SKIPKV_STATUS_COPY_TIMEOUT);
-    *reinterpret_cast<volatile int*>(&ctl->abort_flag) = 1;
-    return false;
-}
-
 template <int kPass>
 __global__ void __launch_bounds__(kTrThreads, 1)
 token_red_kernel(const __grid_constant__ CUtensorMap mapK, int n_slabs, int Hk, int max_cap, const int64_t* slab_off,
                  const int32_t* cap, const int32_t* kv_len, const float* inv_norm, float* z, float* tok_red,
-                 uint32_t* status) {
+                 const Header* hdr) {
     extern __shared__ uint8_t tr_smem_raw[];
     const uint32_t raw = smem_u32(tr_smem_raw);
     uint8_t* At = tr_smem_raw + (((raw + 1023u) & ~1023u) - raw);
@@ -109,31 +95,11 @@ token_red_kernel(const __grid_constant__ CUtensorMap mapK, int n_slabs, int Hk, 
     }
     if (warp == 1) tmem_alloc(&ctl->tmem_base, 128 * kTrGroups);
     pdl_wait();                                          // kv_len and the norms may come from the kernels before
-    {   // prefix of i blocks over slabs (block scan; every thread owns a contiguous block of slabs)
-        const int per = (n_slabs + kTrThreads - 1) / kTrThreads;
-        const int s0 = min(tid * per, n_slabs), s1 = min(s0 + per, n_slabs);
-        uint32_t local = 0;
-        for (int s = s0; s < s1; ++s) local += uint32_t((len_of(s) + 127) >> 7);
-        uint32_t inc = local;
-#pragma unroll
-        for (int d = 1; d < 32; d <<= 1) {
-            const uint32_t x = __shfl_up_sync(0xffffffffu, inc, d);
-            if (lane >= d) inc += x;
-        }
-        if (lane == 31) ctl->wsum[warp] = inc;
-        tc_fence_before();
-        __syncthreads();                                 // also publishes barrier inits and the tmem address
-        tc_fence_after();
-        uint32_t base = 0;
-        for (int w = 0; w < warp; ++w) base += ctl->wsum[w];
-        uint32_t run = base + inc - local;
-        for (int s = s0; s < s1; ++s) {
-            ipref[s] = int(run);
-            run += uint32_t((len_of(s) + 127) >> 7);
-        }
-        if (tid == kTrThreads - 1) ipref[n_slabs] = int(run);
-        __syncthreads();
-    }
+    uint32_t* status = const_cast<uint32_t*>(&hdr->status);
+    const uint32_t limit = load_wait_limit(hdr);
+    tc_fence_before();
+    cta_prefix<kTrThreads>(n_slabs, [&](int s) { return (len_of(s) + 127) >> 7; }, ipref, ctl->wsum);   // i blocks per slab
+    tc_fence_after();
     const uint32_t tmem_base = ctl->tmem_base;
     const int n_items = ipref[n_slabs];
     auto row0_of = [&](int s) { return int(slab_row0(slab_off, cap, Hk, s / Hk, s % Hk)); };
@@ -147,14 +113,14 @@ token_red_kernel(const __grid_constant__ CUtensorMap mapK, int n_slabs, int Hk, 
                 while (ipref[slab + 1] <= item) ++slab;
                 const int NJ = (len_of(slab) + 127) >> 7, row0 = row0_of(slab);
                 const int i0 = (item - ipref[slab]) * 128;
-                if (ic > 0) ok = tr_wait(ctl, &ctl->aempty, (ic - 1) & 1u, status);
+                if (ic > 0) ok = role_wait(&ctl->aempty, (ic - 1) & 1u, limit, &ctl->abort_flag, status);
                 if (!ok) break;
                 mbar_expect_tx(&ctl->afull, kOpBytes);
                 tma_load_2d(At, &mapK, 0, row0 + i0, &ctl->afull);
                 tma_load_2d(At + kOpHalfBytes, &mapK, 64, row0 + i0, &ctl->afull);
                 for (int jb = 0; jb < NJ && ok; ++jb, ++bc) {
                     const int s = bc % kTrStages;
-                    if (bc >= kTrStages) ok = tr_wait(ctl, &ctl->bempty[s], ((bc / kTrStages) - 1) & 1u, status);
+                    if (bc >= kTrStages) ok = role_wait(&ctl->bempty[s], ((bc / kTrStages) - 1) & 1u, limit, &ctl->abort_flag, status);
                     if (!ok) break;
                     uint8_t* dst = Bt + size_t(s) * kOpBytes;
                     mbar_expect_tx(&ctl->bfull[s], kOpBytes);
@@ -176,11 +142,11 @@ token_red_kernel(const __grid_constant__ CUtensorMap mapK, int n_slabs, int Hk, 
             for (int item = cta; item < n_items && ok; item += G, ++ic) {
                 while (ipref[slab + 1] <= item) ++slab;
                 const int NJ = (len_of(slab) + 127) >> 7;
-                ok = tr_wait(ctl, &ctl->afull, ic & 1u, status);
+                ok = role_wait(&ctl->afull, ic & 1u, limit, &ctl->abort_flag, status);
                 for (int jb = 0; jb < NJ && ok; ++jb, ++bc) {
                     const int st = bc % kTrStages, s = bc % kTrGroups;
-                    ok = tr_wait(ctl, &ctl->bfull[st], (bc / kTrStages) & 1u, status);
-                    if (ok && bc >= kTrGroups) ok = tr_wait(ctl, &ctl->tempty[s], ((bc / kTrGroups) - 1) & 1u, status);
+                    ok = role_wait(&ctl->bfull[st], (bc / kTrStages) & 1u, limit, &ctl->abort_flag, status);
+                    if (ok && bc >= kTrGroups) ok = role_wait(&ctl->tempty[s], ((bc / kTrGroups) - 1) & 1u, limit, &ctl->abort_flag, status);
                     if (!ok) break;
                     tc_fence_after();
                     umma_tile_128x128x128(tmem_base + s * 128, a, smem_u32(Bt + size_t(st) * kOpBytes), false);
@@ -221,7 +187,7 @@ token_red_kernel(const __grid_constant__ CUtensorMap mapK, int n_slabs, int Hk, 
                     named_bar_sync(1 + grp, 128);
                 }
                 if (ok) {
-                    ok = tr_wait(ctl, &ctl->tfull[grp], (bc / kTrGroups) & 1u, status);
+                    ok = role_wait(&ctl->tfull[grp], (bc / kTrGroups) & 1u, limit, &ctl->abort_flag, status);
                     ok = __all_sync(0xffffffffu, ok);
                 }
                 if (!ok) continue;                               // keeps the barrier pattern uniform
@@ -292,7 +258,7 @@ extern "C" int skipkv_token_redundancy(const skipkv_shape* shape, const skipkv_p
     if (reinterpret_cast<uintptr_t>(K) & 15) return SKIPKV_ERR_INVALID_ARG;
     const WsLayout L = make_layout(*shape);
     uint8_t* w = static_cast<uint8_t*>(ws);
-    uint32_t* status = &reinterpret_cast<Header*>(w + L.header)->status;
+    const Header* hdr = reinterpret_cast<const Header*>(w + L.header);
     float* inv_norm = reinterpret_cast<float*>(w + L.tr_inv);
     float* z = reinterpret_cast<float*>(w + L.tr_z);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -311,9 +277,9 @@ extern "C" int skipkv_token_redundancy(const skipkv_shape* shape, const skipkv_p
     SKIPKV_CUDA(cudaFuncSetAttribute(token_red_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
     SKIPKV_CUDA(launch_dependent(token_red_kernel<1>, dim3(grid), dim3(kTrThreads), smem, st, mapK, int(L.slabs), Hk,
                                  int(shape->max_cap), shape->slab_off, shape->cap, kv_len, static_cast<const float*>(inv_norm),
-                                 z, tok_red, status));
+                                 z, tok_red, hdr));
     SKIPKV_CUDA(launch_dependent(token_red_kernel<2>, dim3(grid), dim3(kTrThreads), smem, st, mapK, int(L.slabs), Hk,
                                  int(shape->max_cap), shape->slab_off, shape->cap, kv_len, static_cast<const float*>(inv_norm),
-                                 z, tok_red, status));
+                                 z, tok_red, hdr));
     return SKIPKV_OK;
 }
