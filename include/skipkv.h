@@ -100,6 +100,11 @@ int skipkv_workspace_init(const skipkv_shape* shape, void* ws, void* stream);
  * set again; it is read by the kernels enqueued after this call on `stream`.  ws: device. */
 int skipkv_set_wait_limit(void* ws, uint32_t polls, void* stream);
 
+/* Self-check of the time-out path: enqueues one warp that waits, bounded by the workspace's wait limit, for an
+ * event that never happens; when the wait runs out it records SKIPKV_STATUS_COPY_TIMEOUT like any kernel of this
+ * library would, and returns.  Set a small limit first (with the default it spins for seconds).  ws: device. */
+int skipkv_wait_probe(void* ws, void* stream);
+
 /* Read and clear the device status word.  Synchronises `stream`.  *status_bits (host,
  * nullable) receives the SKIPKV_STATUS_* bits; returns SKIPKV_ERR_TIMEOUT if a wait ran out. */
 int skipkv_status(void* ws, void* stream, uint32_t* status_bits);

@@ -24,7 +24,7 @@ SYMBOLS = ["skipkv_workspace_bytes", "skipkv_workspace_init", "skipkv_status", "
            "skipkv_append", "skipkv_decode_attn_static", "skipkv_table_step", "skipkv_score_table",
            "skipkv_select_fill", "skipkv_compact_fill", "skipkv_token_redundancy",
            "skipkv_append_step", "skipkv_decode_attn_paged",
-           "skipkv_decode_step", "skipkv_set_wait_limit"]
+           "skipkv_decode_step", "skipkv_set_wait_limit", "skipkv_wait_probe"]
 
 
 class SkipKVError(RuntimeError):
@@ -150,6 +150,10 @@ def skipkv_decode_attn(shape, q, K, V, kv_len, out, hidden, steer_vec, alpha, fl
 
 def skipkv_set_wait_limit(ws, polls: int, stream=None) -> None:
     _check(lib().skipkv_set_wait_limit(_ptr(ws), C.c_uint32(polls), _stream(stream)), "skipkv_set_wait_limit")
+
+
+def skipkv_wait_probe(ws, stream=None) -> None:
+    _check(lib().skipkv_wait_probe(_ptr(ws), _stream(stream)), "skipkv_wait_probe")
 
 
 def skipkv_steer(batch, d_model, hidden, steer_vec, alpha, flag, stream=None) -> None:

@@ -99,6 +99,16 @@ int check_shape(const skipkv_shape* s) {
 
 __global__ void ws_set_word_kernel(uint32_t* p, uint32_t v) { *p = v; }
 
+// One warp waits, with the workspace's wait limit, for a barrier phase that nothing will ever complete.
+__global__ void __launch_bounds__(32) wait_probe_kernel(Header* hdr) {
+    __shared__ __align__(8) uint64_t bar;
+    if (threadIdx.x == 0) { mbar_init(&bar, 1); mbar_fence_init(); }
+    __syncwarp();
+    const uint32_t limit = load_wait_limit(hdr);
+    const bool ok = mbar_wait(&bar, 0u, limit);
+    if (!ok && threadIdx.x == 0) atomicOr(&hdr->status, SKIPKV_STATUS_COPY_TIMEOUT);
+}
+
 __global__ void ws_clear_kernel(uint32_t* p, size_t n_words) {
     for (size_t i = blockIdx.x * size_t(blockDim.x) + threadIdx.x; i < n_words; i += size_t(gridDim.x) * blockDim.x)
         p[i] = 0u;
@@ -138,6 +148,13 @@ int skipkv_workspace_init(const skipkv_shape* shape, void* ws, void* stream) {
 int skipkv_set_wait_limit(void* ws, uint32_t polls, void* stream) {
     if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255)) return SKIPKV_ERR_WORKSPACE;
     ws_set_word_kernel<<<1, 1, 0, static_cast<cudaStream_t>(stream)>>>(&static_cast<Header*>(ws)->wait_limit, polls);
+    SKIPKV_CUDA(cudaGetLastError());
+    return SKIPKV_OK;
+}
+
+int skipkv_wait_probe(void* ws, void* stream) {
+    if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255)) return SKIPKV_ERR_WORKSPACE;
+    wait_probe_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(static_cast<Header*>(ws));
     SKIPKV_CUDA(cudaGetLastError());
     return SKIPKV_OK;
 }

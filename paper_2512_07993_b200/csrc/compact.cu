@@ -238,9 +238,10 @@ compact_move_kernel(int n_slabs, int Hk, int max_sent, const int64_t* slab_off, 
     __shared__ __align__(8) uint64_t bar;
     __shared__ int s_red[kMoveThreads / 32];
     __shared__ uint32_t s_ticket;
+    __shared__ int s_abort;                            // a wait of this CTA ran out: it takes no further segment
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
-    if (tid == 0) { mbar_init(&bar, 1); mbar_fence_init(); }
+    if (tid == 0) { mbar_init(&bar, 1); mbar_fence_init(); s_abort = 0; }
     // everything below reads what the plan kernel wrote: wait until that grid has completed and its writes are visible
     pdl_wait();
     // every CTA derives the scheduler bound: the largest segment count of any slab
@@ -259,6 +260,7 @@ compact_move_kernel(int n_slabs, int Hk, int max_sent, const int64_t* slab_off, 
 
     for (;;) {
         __syncthreads();                               // s_ticket / smem free for the next round
+        if (s_abort) break;                            // (read by every thread after the barrier: a uniform exit)
         if (tid == 0) s_ticket = atomicAdd(&hdr->compact_ticket, 1u);
         __syncthreads();
         const uint32_t T = s_ticket;
@@ -341,6 +343,11 @@ compact_move_kernel(int n_slabs, int Hk, int max_sent, const int64_t* slab_off, 
                                  uint32_t(pe - ps) * kRowBytes);
                 }
                 bulk_commit();
+            } else {
+                // A wait ran out (flagged above): the stores of this segment are skipped and this CTA stops.  Its own
+                // loads may still be in flight towards its shared memory, and they must land before it retires.
+                mbar_wait(&bar, phase, 1u << 20);
+                if (lane == 0) s_abort = 1;
             }
             bulk_wait_read_all();                      // shared memory may be refilled
         }

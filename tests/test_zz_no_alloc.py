@@ -6,12 +6,14 @@ skipkv_decode_attn.  The static variant keeps its scratch in a fixed array insid
 Here it is called through the C ABI twice in a row (the array keeps the previous call's
 contents, so the second call checks that what must start at zero is cleared) and compared with
 the workspace-based entry point on the same inputs, within the decode-attention tolerance of the
-parity tests.  This file is collected last so that a failure here cannot hide another test.
+parity tests, and, on two slabs, directly with the CPU oracle's attention.  This file is collected last
+so that a failure here cannot hide another test.
 """
 import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2512_07993_b200 import workloads as W
 
 pytestmark = pytest.mark.gpu
@@ -59,6 +61,16 @@ def test_static_scratch_decode_matches_workspace_decode_twice():
         assert int(status.item()) == 0
         assert torch.isfinite(got.float()).all()
         assert rel_err(got, want) <= TOL, call
+        # and against the oracle itself, on two slabs with the lengths of this call
+        g = cfg.group
+        Kb, Vb, qb = W.bf16_bits(L["K"]), W.bf16_bits(L["V"]), W.bf16_bits(L["q"])
+        lens = D.kv_len.cpu().numpy()
+        for (b, h) in [(0, 3), (1, 6)]:
+            rows = W.slab_rows(L, b, h)
+            n = int(lens[b, h])
+            _, o64 = oracle.decode_attn(qb[b, h * g:(h + 1) * g], Kb[rows][:n], Vb[rows][:n], n)
+            mine = got[b, h * g:(h + 1) * g].float().cpu().numpy().astype(np.float64)
+            assert (np.abs(mine - o64) / np.abs(o64).max(axis=-1, keepdims=True)).max() <= TOL, (call, b, h)
         # the fused steering add is the same bit-exact operation as in the workspace variant
         ref_h = D.hidden.clone()
         B.skipkv_steer(cfg.batch, cfg.d_model, ref_h, D.steer_vec, D.alpha, D.flag)
