@@ -175,18 +175,30 @@ def score_with_table(K_bits, Q_bits, sent_off, sent_id, T, sigma, tau, eps=1e-6)
 
 
 # ------------------------------------------------------------------ exactly-B retention
-def select_fill(score, sent_off, tok_imp, budget, protect_tail):
+def token_final_key(tok_imp, tok_red, sigma):
+    """Per-token key of the cut sentence when a token-level redundancy is given (Section 4.1, Eq. "I_final" with the
+    token-level R of the "Token Redundancy Score" paragraph; the penalty is the same for all tokens of a sentence and
+    drops out of the order): sigma * I - (1 - sigma) * R, each operation rounded to fp32 (the precision in which the
+    order is decided)."""
+    s = np.float32(sigma)
+    return (s * np.asarray(tok_imp, np.float32)).astype(np.float32) - ((np.float32(1) - s) * np.asarray(tok_red, np.float32)).astype(np.float32)
+
+
+def select_fill(score, sent_off, tok_imp, budget, protect_tail, tok_red=None, sigma=None):
     """O12  Selection that retains exactly B tokens (Section 4.1: tokens are evicted in increasing
     order of the final score until the cache meets the budget).  Whole sentences are kept in rank
     order as in O5; the first sentence that does not fit (the cut sentence) then gives up only its
     lowest-scoring tokens: redundancy and penalty are the same for all tokens of a sentence, so
     inside it the final-score order is the token-importance order.  Its `slack = B - kept` tokens of
-    largest tok_imp survive (equal values: the earlier token first).
+    largest tok_imp survive (equal values: the earlier token first).  With tok_red (token-level redundancy, O14)
+    the tokens of the cut sentence are ordered by token_final_key instead.
 
     score fp32 [S], sent_off int32 [S+1], tok_imp fp32 [N].  Returns (keep uint8 [S] with 1 = whole
     sentence kept, 2 = cut sentence partly kept; tok_keep uint8 [N]; new_len)."""
     score = np.asarray(score, np.float32); sent_off = np.asarray(sent_off, np.int64)
     tok_imp = np.asarray(tok_imp, np.float32)
+    if tok_red is not None:
+        tok_imp = token_final_key(tok_imp, tok_red, sigma)
     S = len(sent_off) - 1
     total = int(sent_off[S]) if S > 0 else 0
     keep = np.zeros(S, np.uint8); tok_keep = np.zeros(total, np.uint8)

@@ -534,6 +534,35 @@ def test_o12_hand_example():
     assert keep.all() and tk.all() and nl == 14
 
 
+def test_o12_token_level_redundancy_orders_the_cut_sentence():
+    """With a token-level redundancy the cut sentence gives up its tokens in the order of
+    sigma * I - (1 - sigma) * R (Eq. "I_final" per token): hand example where the redundancy overturns the
+    importance order, the limits sigma = 1 (importance alone) and R constant (importance alone again)."""
+    lens = [2, 5]
+    off = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    score = np.array([0.9, 0.1], np.float32)                     # sentence 0 first, sentence 1 is cut
+    imp = np.array([0, 0, 0.50, 0.40, 0.30, 0.20, 0.10], np.float32)
+    red = np.array([0, 0, 0.90, 0.10, 0.80, 0.00, 0.05], np.float32)
+    # sigma = 0.5: keys 0.5*I - 0.5*R = -0.20, 0.15, -0.25, 0.10, 0.025 -> order of tokens 3, 5, 6, 2, 4
+    keep, tk, nl = oracle.select_fill(score, off, imp, 4, 0, tok_red=red, sigma=0.5)
+    assert np.array_equal(keep, [1, 2]) and nl == 4
+    assert np.array_equal(np.nonzero(tk)[0], [0, 1, 3, 5])
+    keep, tk, nl = oracle.select_fill(score, off, imp, 6, 0, tok_red=red, sigma=0.5)
+    assert np.array_equal(np.nonzero(tk)[0], [0, 1, 2, 3, 5, 6])   # the most redundant token (4) goes first
+    # sigma = 1: the redundancy has no weight
+    k1, t1, _ = oracle.select_fill(score, off, imp, 4, 0, tok_red=red, sigma=1.0)
+    k0, t0, _ = oracle.select_fill(score, off, imp, 4, 0)
+    assert np.array_equal(t1, t0) and np.array_equal(np.nonzero(t0)[0], [0, 1, 2, 3])
+    # a constant redundancy shifts every key alike (in exact arithmetic; here with values that stay exact in fp32)
+    kc, tc, _ = oracle.select_fill(score, off, imp, 4, 0, tok_red=np.full(7, 0.25, np.float32), sigma=0.5)
+    assert np.array_equal(tc, t0)
+    # the key itself: each operation rounded to fp32
+    key = oracle.token_final_key(imp, red, 0.5)
+    assert key.dtype == np.float32
+    want = [np.float32(np.float32(0.5) * i) - np.float32(np.float32(0.5) * r) for i, r in zip(imp, red)]
+    assert np.array_equal(key, np.array(want, np.float32))
+
+
 def test_o12_random_properties():
     r = np.random.default_rng(7)
     for trial in range(60):
