@@ -262,6 +262,19 @@ int skipkv_select_fill(const skipkv_shape* shape, const skipkv_params* params, c
                        const float* tok_imp, const int32_t* sent_off, const int32_t* n_sent, uint8_t* keep,
                        uint8_t* tok_keep, int32_t* kept_idx, int32_t* n_kept, int32_t* new_len, void* ws,
                        void* stream);
+
+/*
+ * skipkv_select_fill_red -- skipkv_select_fill with the token-level redundancy of Section 4.1 ("Token Redundancy
+ * Score" paragraph, as computed by skipkv_token_redundancy) deciding inside the cut sentence: its tokens leave in
+ * increasing order of sigma * tok_imp[t] - (1 - sigma) * tok_red[t], Eq. "I_final" per token (the penalty is the same
+ * for all tokens of a sentence and does not change their order).  The key is formed in fp32, every operation rounded
+ * to nearest; equal keys: the earlier token stays first.  tok_red: device fp32, one value per cache row with the row
+ * indexing of K (read only).  Everything else as skipkv_select_fill.
+ */
+int skipkv_select_fill_red(const skipkv_shape* shape, const skipkv_params* params, const float* sent_score,
+                           const float* tok_imp, const float* tok_red, const int32_t* sent_off,
+                           const int32_t* n_sent, uint8_t* keep, uint8_t* tok_keep, int32_t* kept_idx,
+                           int32_t* n_kept, int32_t* new_len, void* ws, void* stream);
 int skipkv_compact_fill(const skipkv_shape* shape, void* K, void* V, const uint8_t* keep,
                         const uint8_t* tok_keep, int32_t* sent_off, int32_t* sent_id, int32_t* n_sent,
                         int32_t* kv_len, int32_t* index_map, void* ws, void* stream);

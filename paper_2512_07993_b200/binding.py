@@ -24,7 +24,7 @@ SYMBOLS = ["skipkv_workspace_bytes", "skipkv_workspace_init", "skipkv_status", "
            "skipkv_append", "skipkv_decode_attn_static", "skipkv_table_step", "skipkv_score_table",
            "skipkv_select_fill", "skipkv_compact_fill", "skipkv_token_redundancy",
            "skipkv_append_step", "skipkv_decode_attn_paged",
-           "skipkv_decode_step", "skipkv_set_wait_limit", "skipkv_wait_probe"]
+           "skipkv_decode_step", "skipkv_set_wait_limit", "skipkv_wait_probe", "skipkv_select_fill_red"]
 
 
 class SkipKVError(RuntimeError):
@@ -197,6 +197,16 @@ def skipkv_select_fill(shape, params, sent_score, tok_imp, sent_off, n_sent, kee
                                     _ptr(n_sent, torch.int32), _ptr(keep, torch.uint8), _ptr(tok_keep, torch.uint8),
                                     _ptr(kept_idx, torch.int32), _ptr(n_kept, torch.int32),
                                     _ptr(new_len, torch.int32), _ptr(ws), _stream(stream)), "skipkv_select_fill")
+
+
+def skipkv_select_fill_red(shape, params, sent_score, tok_imp, tok_red, sent_off, n_sent, keep, tok_keep, kept_idx,
+                           n_kept, new_len, ws, stream=None) -> None:
+    _check(lib().skipkv_select_fill_red(C.byref(shape), C.byref(params), _ptr(sent_score, torch.float32),
+                                        _ptr(tok_imp, torch.float32), _ptr(tok_red, torch.float32),
+                                        _ptr(sent_off, torch.int32), _ptr(n_sent, torch.int32), _ptr(keep, torch.uint8),
+                                        _ptr(tok_keep, torch.uint8), _ptr(kept_idx, torch.int32),
+                                        _ptr(n_kept, torch.int32), _ptr(new_len, torch.int32), _ptr(ws),
+                                        _stream(stream)), "skipkv_select_fill_red")
 
 
 def skipkv_compact_fill(shape, K, V, keep, tok_keep, sent_off, sent_id, n_sent, kv_len, index_map, ws,

@@ -77,14 +77,16 @@ struct SweepArgs {
 };
 
 // ---- sweep 1 epilogue: one accumulator (128 tokens) folded into the running (max, sum) of a row
+// (The loop over the four 32-column pieces is kept rolled, here and in imp_fold for four heads per group: the epilogue
+// code is fetched again for every tile, and unrolled it stalls on instruction fetch more than the loop costs.)
 template <bool kMasked>
 __device__ __forceinline__ void lse_fold(uint32_t taddr, int valid, float scale, float& m, float& l) {
-#pragma unroll
-    for (int ch = 0; ch < 4; ++ch) {
-        if (kMasked && ch * 32 >= valid) break;
+    const int nch = kMasked ? (valid + 31) >> 5 : 4;
+#pragma unroll 1
+    for (int ch = 0; ch < nch; ++ch) {
         float v[32];
         tmem_ld32(taddr + ch * 32, v);
-        if (kMasked) {
+        if (kMasked && ch * 32 + 32 > valid) {
 #pragma unroll
             for (int j = 0; j < 32; ++j)
                 if (ch * 32 + j >= valid) v[j] = -INFINITY;
@@ -111,6 +113,31 @@ __device__ __forceinline__ void lse_fold(uint32_t taddr, int valid, float scale,
 template <int kN>
 __device__ __forceinline__ float imp_fold(uint32_t taddr, const float* neg_lse, int wvalid, float scale) {
     constexpr int WB = 128 / kN;
+    if constexpr (kN == 4) {
+        float b4[32];
+#pragma unroll
+        for (int j = 0; j < 32; ++j) b4[j] = -INFINITY;
+#pragma unroll 1
+        for (int q = 0; q < 4; ++q) {
+            float v[32];
+            tmem_ld32(taddr + q * 32, v);
+#pragma unroll
+            for (int j4 = 0; j4 < 32; j4 += 4) {
+                const float4 nl = *reinterpret_cast<const float4*>(neg_lse + q * 32 + j4);
+                b4[j4 + 0] = fmaxf(b4[j4 + 0], fmaf(v[j4 + 0], scale, nl.x));
+                b4[j4 + 1] = fmaxf(b4[j4 + 1], fmaf(v[j4 + 1], scale, nl.y));
+                b4[j4 + 2] = fmaxf(b4[j4 + 2], fmaf(v[j4 + 2], scale, nl.z));
+                b4[j4 + 3] = fmaxf(b4[j4 + 3], fmaf(v[j4 + 3], scale, nl.w));
+            }
+        }
+        float t0 = 0.f, t1 = 0.f;
+#pragma unroll
+        for (int j = 0; j < 32; j += 2) {
+            t0 += (j < wvalid) ? ex2f(b4[j]) : 0.f;
+            t1 += (j + 1 < wvalid) ? ex2f(b4[j + 1]) : 0.f;
+        }
+        return t0 + t1;
+    }
     float best[WB];
     float total = 0.f;
 #pragma unroll

@@ -49,6 +49,8 @@ __device__ __forceinline__ uint32_t block_excl(uint32_t v, uint32_t* wsum, uint3
 // keep = 2.  tok_imp is indexed by cache row when from_rows is set, else [slab][max_cap].
 struct FillArgs {
     const float* tok_imp;
+    const float* tok_red;      // nullable, one value per cache row: the cut sentence's tokens are then ordered by
+    float sigma;               // sigma * tok_imp - (1 - sigma) * tok_red (each operation rounded to fp32)
     uint8_t* tok_keep;
     const int64_t* slab_off;
     const int32_t* cap;
@@ -143,11 +145,17 @@ select_kernel(int max_sent, int P, int budget, int protect_tail, const float* se
         const size_t row0 = slab_row0(fill.slab_off, fill.cap, fill.Hk, b, h);
         const float* imp = fill.from_rows ? fill.tok_imp + row0 + cb : fill.tok_imp + size_t(slab) * fill.max_cap + cb;
         uint8_t* tk = fill.tok_keep + row0 + cb;
+        const float* red = fill.tok_red ? fill.tok_red + row0 + cb : nullptr;
+        const float w_red = __fsub_rn(1.f, fill.sigma);
+        auto key = [&](int u) {
+            const float i = __ldg(imp + u);
+            return red ? __fsub_rn(__fmul_rn(fill.sigma, i), __fmul_rn(w_red, __ldg(red + u))) : i;
+        };
         for (int t = tid; t < len; t += kSelThreads) {   // rank by counting: tokens that come before t in the order
-            const float mine = imp[t];
+            const float mine = key(t);
             int rank = 0;
             for (int u = 0; u < len; ++u) {
-                const float other = __ldg(imp + u);
+                const float other = key(u);
                 rank += (other > mine || (other == mine && u < t)) ? 1 : 0;
             }
             tk[t] = rank < slack ? 1 : 0;
@@ -216,17 +224,36 @@ extern "C" int skipkv_select(const skipkv_shape* shape, const skipkv_params* par
                        stream);
 }
 
-extern "C" int skipkv_select_fill(const skipkv_shape* shape, const skipkv_params* params, const float* sent_score,
-                                  const float* tok_imp, const int32_t* sent_off, const int32_t* n_sent, uint8_t* keep,
-                                  uint8_t* tok_keep, int32_t* kept_idx, int32_t* n_kept, int32_t* new_len, void* ws,
-                                  void* stream) {
-    if (!tok_keep) return SKIPKV_ERR_INVALID_ARG;
+static int select_fill_impl(const skipkv_shape* shape, const skipkv_params* params, const float* sent_score,
+                            const float* tok_imp, const float* tok_red, const int32_t* sent_off, const int32_t* n_sent,
+                            uint8_t* keep, uint8_t* tok_keep, int32_t* kept_idx, int32_t* n_kept, int32_t* new_len, void* ws,
+                            void* stream) {
+    if (!tok_keep || !params) return SKIPKV_ERR_INVALID_ARG;
     if (int rc = check_shape(shape)) return rc;
     if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255)) return SKIPKV_ERR_WORKSPACE;
     FillArgs fill{};
     fill.tok_keep = tok_keep;
+    fill.tok_red = tok_red;
+    fill.sigma = params->sigma;
     fill.slab_off = shape->slab_off; fill.cap = shape->cap; fill.Hk = shape->n_kv_heads; fill.max_cap = shape->max_cap;
     if (tok_imp) { fill.tok_imp = tok_imp; fill.from_rows = 1; }
     else { fill.tok_imp = reinterpret_cast<const float*>(static_cast<uint8_t*>(ws) + make_layout(*shape).sc_tokimp); }
     return select_impl(shape, params, sent_score, sent_off, n_sent, keep, kept_idx, n_kept, new_len, fill, ws, stream);
+}
+
+extern "C" int skipkv_select_fill(const skipkv_shape* shape, const skipkv_params* params, const float* sent_score,
+                                  const float* tok_imp, const int32_t* sent_off, const int32_t* n_sent, uint8_t* keep,
+                                  uint8_t* tok_keep, int32_t* kept_idx, int32_t* n_kept, int32_t* new_len, void* ws,
+                                  void* stream) {
+    return select_fill_impl(shape, params, sent_score, tok_imp, nullptr, sent_off, n_sent, keep, tok_keep, kept_idx, n_kept,
+                            new_len, ws, stream);
+}
+
+extern "C" int skipkv_select_fill_red(const skipkv_shape* shape, const skipkv_params* params, const float* sent_score,
+                                      const float* tok_imp, const float* tok_red, const int32_t* sent_off,
+                                      const int32_t* n_sent, uint8_t* keep, uint8_t* tok_keep, int32_t* kept_idx,
+                                      int32_t* n_kept, int32_t* new_len, void* ws, void* stream) {
+    if (!tok_red) return SKIPKV_ERR_INVALID_ARG;
+    return select_fill_impl(shape, params, sent_score, tok_imp, tok_red, sent_off, n_sent, keep, tok_keep, kept_idx, n_kept,
+                            new_len, ws, stream);
 }

@@ -140,6 +140,40 @@ def test_fill_against_oracle_scores():
     assert excused <= 2
 
 
+def test_select_fill_with_token_level_redundancy():
+    """skipkv_token_redundancy feeds skipkv_select_fill_red: inside the cut sentence the tokens are ordered by
+    sigma * tok_imp - (1 - sigma) * tok_red.  The oracle's rule applied to the GPU's own scores, importances and
+    redundancies is reproduced bit for bit; sigma = 0.01 so that the (small) spread of the redundancy decides."""
+    cfg = CASES["ragged"]()
+    L, D, B = device_layer(cfg)
+    params = B.make_params(0.01, 0.95, 1e-6, cfg.budget, cfg.window)
+    D.params = params
+    D.score()
+    tok_red = torch.zeros(D.K.shape[0], dtype=torch.float32, device="cuda")
+    B.skipkv_token_redundancy(D.shape, D.params, D.K, D.kv_len, tok_red, D.ws)
+    B.skipkv_select_fill_red(D.shape, D.params, D.sent_score, D.tok_imp, tok_red, D.sent_off, D.n_sent, D.keep, D.tok_keep,
+                             D.kept_idx, D.n_kept, D.new_len, D.ws)
+    torch.cuda.synchronize()
+    assert D.status() == 0
+    sc, tok, red = D.sent_score.cpu().numpy(), D.tok_imp.cpu().numpy(), tok_red.cpu().numpy()
+    keep, tk, new_len = D.keep.cpu().numpy(), D.tok_keep.cpu().numpy(), D.new_len.cpu().numpy()
+    n_cut = differs = 0
+    for b in range(cfg.batch):
+        for h in range(cfg.n_kv_heads):
+            rows = W.slab_rows(L, b, h)
+            N, S = int(L["kv_len"][b, h]), int(L["n_sent"][b, h])
+            off = L["sent_off"][b, h, :S + 1]
+            k_ref, t_ref, nl = oracle.select_fill(sc[b, h, :S], off, tok[rows][:N], cfg.budget, cfg.window,
+                                                  tok_red=red[rows][:N], sigma=float(np.float32(0.01)))
+            assert np.array_equal(keep[b, h, :S], k_ref) and int(new_len[b, h]) == nl
+            _, t_imp, _ = oracle.select_fill(sc[b, h, :S], off, tok[rows][:N], cfg.budget, cfg.window)
+            for c in np.nonzero(k_ref == 2)[0]:
+                n_cut += 1
+                assert np.array_equal(tk[rows][off[c]:off[c + 1]], t_ref[off[c]:off[c + 1]]), f"tok_keep ({b},{h})"
+                differs += int(not np.array_equal(t_ref[off[c]:off[c + 1]], t_imp[off[c]:off[c + 1]]))
+    assert n_cut > 0 and differs > 0          # the redundancy did change some cut sentence's survivors
+
+
 def test_compact_fill_several_partial_sentences():
     """Hand-made selections: up to four partly kept sentences per slab, among them one longer than a packing
     pass, one with every token flagged, one with none (it disappears), and neighbours that are both partial."""
