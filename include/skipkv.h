@@ -13,7 +13,10 @@
  * and, beside them, the generation-space lookup table of the sentence penalty (skipkv_table_step)
  * with the score variant that reads it (skipkv_score_table), and the variants of select and compact that
  * retain exactly B tokens (skipkv_select_fill, skipkv_compact_fill), and the redundancy term over single
- * tokens (skipkv_token_redundancy).
+ * tokens (skipkv_token_redundancy) with the selection that uses it (skipkv_select_fill_red), the per-step append
+ * (skipkv_append, skipkv_append_step) and its fusion with the attention (skipkv_decode_step), and the same steps
+ * over a paged cache (skipkv_score_paged, skipkv_compact_paged, skipkv_decode_attn_paged,
+ * skipkv_decode_step_paged).
  *
  * Conventions
  *   - Every pointer marked "device" is a CUDA device pointer; "host" is ordinary memory.
@@ -96,8 +99,9 @@ int skipkv_workspace_init(const skipkv_shape* shape, void* ws, void* stream);
 
 /* Set how many times a bounded device wait polls before it gives up and records SKIPKV_STATUS_*_TIMEOUT in the
  * status word (every wait inside the kernels is bounded: a copy that never lands, or a hand-off another thread
- * block never makes, ends the wait instead of hanging the GPU).  polls = 0 restores the default (about four million.  The value lives in the workspace and is kept by skipkv_workspace_init... until it is
- * set again; it is read by the kernels enqueued after this call on `stream`.  ws: device. */
+ * block never makes, ends the wait instead of hanging the GPU).  polls = 0 restores the default (about four
+ * million polls, seconds of waiting).  The value lives in the workspace, survives skipkv_workspace_init, and is
+ * read by the kernels enqueued after this call on `stream`.  ws: device. */
 int skipkv_set_wait_limit(void* ws, uint32_t polls, void* stream);
 
 /* Self-check of the time-out path: enqueues one warp that waits, bounded by the workspace's wait limit, for an
@@ -327,6 +331,31 @@ int skipkv_decode_attn_paged(const skipkv_shape* shape, const void* q, const voi
                              void* ws, void* stream);
 
 /*
+ * skipkv_score_paged -- skipkv_score over the paged cache of skipkv_decode_attn_paged (same pool, block table and
+ * page size).  Only K is read.  tok_imp (nullable) is laid out per slab with a stride of max_pages *
+ * SKIPKV_PAGE_ROWS floats: tok_imp[(b*Hk + h) * max_pages * SKIPKV_PAGE_ROWS + t].  Requires
+ * max_pages * SKIPKV_PAGE_ROWS <= max_cap + SKIPKV_PAGE_ROWS - 1 (the workspace is sized from max_cap) and
+ * shape->total_rows = rows of the pool.  shape->slab_off is not used.  Every other argument and every output as
+ * skipkv_score; the two give bit-identical results for the same rows.
+ */
+int skipkv_score_paged(const skipkv_shape* shape, const skipkv_params* params, const void* K_pages,
+                       const int32_t* block_table, int32_t max_pages, const void* q_win, const int32_t* kv_len,
+                       const int32_t* sent_off, const int32_t* n_sent, float* tok_imp, float* sent_imp,
+                       float* sent_red, float* sent_lam, float* sent_score, void* ws, void* stream);
+
+/*
+ * skipkv_compact_paged -- skipkv_compact over the paged cache: the surviving rows of slab (b, h) are packed to the
+ * front of the slab's own pages, in the order of its block table (row t of the packed slab is row
+ * t % SKIPKV_PAGE_ROWS of page block_table[b][h][t / SKIPKV_PAGE_ROWS]); the block table itself is not changed, so
+ * the pages behind the new kv_len are free for the caller to return to its pool.  Two slabs must not share a
+ * page.  index_map (nullable) has a stride of max_pages * SKIPKV_PAGE_ROWS per slab, like tok_imp of
+ * skipkv_score_paged.  Everything else, and the resulting rows, tables and lengths, as skipkv_compact.
+ */
+int skipkv_compact_paged(const skipkv_shape* shape, void* K_pages, void* V_pages, const int32_t* block_table,
+                         int32_t max_pages, const uint8_t* keep, int32_t* sent_off, int32_t* sent_id,
+                         int32_t* n_sent, int32_t* kv_len, int32_t* index_map, void* ws, void* stream);
+
+/*
  * skipkv_decode_step -- one decode step of Algorithm 2 for one layer in a single launch: skipkv_append_step
  * followed by skipkv_decode_attn (attention over the cache including the new row, steering add), fused.
  * The new K/V row of (b, h) is written at kv_len_in[b][h] and attended to; the range list and the observation
@@ -341,6 +370,19 @@ int skipkv_decode_step(const skipkv_shape* shape, const void* q, const void* k_n
                        int32_t* sent_id, int32_t* n_sent, const uint8_t* new_sent, const int32_t* gen_id,
                        void* q_win, int32_t slot, void* out, void* hidden, const void* steer_vec,
                        const float* alpha, const uint8_t* flag, void* ws, void* stream);
+
+/*
+ * skipkv_decode_step_paged -- skipkv_decode_step over the paged cache: the new row of (b, h) goes to row
+ * kv_len_in % SKIPKV_PAGE_ROWS of page block_table[b][h][kv_len_in / SKIPKV_PAGE_ROWS], which the caller must have
+ * assigned before the call (a slab needs (kv_len_in + 1) rows' worth of pages; room is
+ * min(cap[b], max_pages * SKIPKV_PAGE_ROWS)).  Everything else as skipkv_decode_step.
+ */
+int skipkv_decode_step_paged(const skipkv_shape* shape, const void* q, const void* k_new, const void* v_new,
+                             void* K_pages, void* V_pages, const int32_t* block_table, int32_t max_pages,
+                             const int32_t* kv_len_in, int32_t* kv_len_out, int32_t* sent_off, int32_t* sent_id,
+                             int32_t* n_sent, const uint8_t* new_sent, const int32_t* gen_id, void* q_win,
+                             int32_t slot, void* out, void* hidden, const void* steer_vec, const float* alpha,
+                             const uint8_t* flag, void* ws, void* stream);
 
 /*
  * skipkv_decode_attn_static -- skipkv_decode_attn for callers that cannot allocate device

@@ -24,7 +24,8 @@ SYMBOLS = ["skipkv_workspace_bytes", "skipkv_workspace_init", "skipkv_status", "
            "skipkv_append", "skipkv_decode_attn_static", "skipkv_table_step", "skipkv_score_table",
            "skipkv_select_fill", "skipkv_compact_fill", "skipkv_token_redundancy",
            "skipkv_append_step", "skipkv_decode_attn_paged",
-           "skipkv_decode_step", "skipkv_set_wait_limit", "skipkv_wait_probe", "skipkv_select_fill_red"]
+           "skipkv_decode_step", "skipkv_set_wait_limit", "skipkv_wait_probe", "skipkv_select_fill_red",
+           "skipkv_score_paged", "skipkv_compact_paged", "skipkv_decode_step_paged"]
 
 
 class SkipKVError(RuntimeError):
@@ -243,6 +244,44 @@ def skipkv_decode_attn_paged(shape, q, K_pages, V_pages, block_table, max_pages,
                                           _ptr(hidden, torch.bfloat16), _ptr(steer_vec, torch.bfloat16),
                                           _ptr(alpha, torch.float32), _ptr(flag, torch.uint8), _ptr(ws),
                                           _stream(stream)), "skipkv_decode_attn_paged")
+
+
+def skipkv_score_paged(shape, params, K_pages, block_table, max_pages, q_win, kv_len, sent_off, n_sent, tok_imp,
+                       sent_imp, sent_red, sent_lam, sent_score, ws, stream=None) -> None:
+    _check(lib().skipkv_score_paged(C.byref(shape), C.byref(params), _ptr(K_pages, torch.bfloat16),
+                                    _ptr(block_table, torch.int32), C.c_int32(max_pages),
+                                    _ptr(q_win, torch.bfloat16), _ptr(kv_len, torch.int32),
+                                    _ptr(sent_off, torch.int32), _ptr(n_sent, torch.int32),
+                                    _ptr(tok_imp, torch.float32), _ptr(sent_imp, torch.float32),
+                                    _ptr(sent_red, torch.float32), _ptr(sent_lam, torch.float32),
+                                    _ptr(sent_score, torch.float32), _ptr(ws), _stream(stream)),
+           "skipkv_score_paged")
+
+
+def skipkv_compact_paged(shape, K_pages, V_pages, block_table, max_pages, keep, sent_off, sent_id, n_sent, kv_len,
+                         index_map, ws, stream=None) -> None:
+    _check(lib().skipkv_compact_paged(C.byref(shape), _ptr(K_pages, torch.bfloat16), _ptr(V_pages, torch.bfloat16),
+                                      _ptr(block_table, torch.int32), C.c_int32(max_pages),
+                                      _ptr(keep, torch.uint8), _ptr(sent_off, torch.int32),
+                                      _ptr(sent_id, torch.int32), _ptr(n_sent, torch.int32),
+                                      _ptr(kv_len, torch.int32), _ptr(index_map, torch.int32), _ptr(ws),
+                                      _stream(stream)), "skipkv_compact_paged")
+
+
+def skipkv_decode_step_paged(shape, q, k_new, v_new, K_pages, V_pages, block_table, max_pages, kv_len_in, kv_len_out,
+                             sent_off, sent_id, n_sent, new_sent, gen_id, q_win, slot, out, hidden, steer_vec, alpha,
+                             flag, ws, stream=None) -> None:
+    _check(lib().skipkv_decode_step_paged(C.byref(shape), _ptr(q, torch.bfloat16), _ptr(k_new, torch.bfloat16),
+                                          _ptr(v_new, torch.bfloat16), _ptr(K_pages, torch.bfloat16),
+                                          _ptr(V_pages, torch.bfloat16), _ptr(block_table, torch.int32),
+                                          C.c_int32(max_pages), _ptr(kv_len_in, torch.int32),
+                                          _ptr(kv_len_out, torch.int32), _ptr(sent_off, torch.int32),
+                                          _ptr(sent_id, torch.int32), _ptr(n_sent, torch.int32),
+                                          _ptr(new_sent, torch.uint8), _ptr(gen_id, torch.int32),
+                                          _ptr(q_win, torch.bfloat16), C.c_int32(slot), _ptr(out, torch.bfloat16),
+                                          _ptr(hidden, torch.bfloat16), _ptr(steer_vec, torch.bfloat16),
+                                          _ptr(alpha, torch.float32), _ptr(flag, torch.uint8), _ptr(ws),
+                                          _stream(stream)), "skipkv_decode_step_paged")
 
 
 def skipkv_decode_step(shape, q, k_new, v_new, K, V, kv_len_in, kv_len_out, sent_off, sent_id, n_sent, new_sent, gen_id,

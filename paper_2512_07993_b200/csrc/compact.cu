@@ -233,7 +233,7 @@ __global__ void __launch_bounds__(kMoveThreads)
 compact_move_kernel(int n_slabs, int Hk, int max_sent, const int64_t* slab_off, const int32_t* cap,
                     __nv_bfloat16* K, __nv_bfloat16* V, int32_t* index_map, Header* hdr, const int32_t* cp_nseg,
                     uint32_t* cp_loaded, const int32_t* cp_nruns, const int32_t* cp_run_src,
-                    const int32_t* cp_run_dst) {
+                    const int32_t* cp_run_dst, const int32_t* block_table, int max_pages) {
     extern __shared__ __align__(1024) uint8_t smem[];
     __shared__ __align__(8) uint64_t bar;
     __shared__ int s_red[kMoveThreads / 32];
@@ -269,8 +269,18 @@ compact_move_kernel(int n_slabs, int Hk, int max_sent, const int64_t* slab_off, 
         const int slab = stream >> 1;
         if (j >= cp_nseg[slab]) continue;
         const int b = slab / Hk, h = slab % Hk;
-        const size_t row0 = slab_row0(slab_off, cap, Hk, b, h);
-        uint8_t* base = reinterpret_cast<uint8_t*>((stream & 1) ? V : K) + row0 * kRowBytes;
+        // contiguous slabs: token t of the slab is row row0 + t; paged cache (128-row pages): row table[t / 128] * 128 + t % 128,
+        // and a copy is cut where its source or its destination crosses a page
+        const int32_t* table = block_table ? block_table + size_t(slab) * max_pages : nullptr;
+        const size_t row0 = table ? size_t(slab) * max_pages * 128 : slab_row0(slab_off, cap, Hk, b, h);   // (paged: index_map rows)
+        uint8_t* tensor = reinterpret_cast<uint8_t*>((stream & 1) ? V : K);
+        uint8_t* base = tensor + (table ? 0 : row0 * kRowBytes);
+        auto row_ptr = [&](int t) {
+            return table ? tensor + (size_t(max(table[t >> 7], 0)) * 128 + (t & 127)) * kRowBytes : base + size_t(t) * kRowBytes;
+        };
+        auto piece_rows = [&](int src, int dst, int left) {      // rows of a copy that stay inside one page on both sides
+            return table ? min(left, min(128 - (src & 127), 128 - (dst & 127))) : left;
+        };
         const int32_t* run_src = cp_run_src + size_t(slab) * max_sent;
         const int32_t* run_dst = cp_run_dst + size_t(slab) * (max_sent + 1);
         const int nruns = cp_nruns[slab];
@@ -302,8 +312,11 @@ compact_move_kernel(int n_slabs, int Hk, int max_sent, const int64_t* slab_off, 
                 const int ps = max(run_dst[r], d0), pe = min(run_dst[r + 1], d1);
                 const int src = run_src[r] + (ps - run_dst[r]);
                 if (src != ps)
-                    bulk_g2s(smem + size_t(ps - d0) * kRowBytes, base + size_t(src) * kRowBytes,
-                             uint32_t(pe - ps) * kRowBytes, &bar);
+                    for (int o = 0; o < pe - ps;) {
+                        const int nr = piece_rows(src + o, ps + o, pe - ps - o);
+                        bulk_g2s(smem + size_t(ps + o - d0) * kRowBytes, row_ptr(src + o), uint32_t(nr) * kRowBytes, &bar);
+                        o += nr;
+                    }
             }
         } else if (index_map != nullptr && (stream & 1) == 0) {
             // dest token k of this segment came from token run_src[r] + (k - run_dst[r])
@@ -339,8 +352,11 @@ compact_move_kernel(int n_slabs, int Hk, int max_sent, const int64_t* slab_off, 
                     const int ps = max(run_dst[r], d0), pe = min(run_dst[r + 1], d1);
                     const int src = run_src[r] + (ps - run_dst[r]);
                     if (src != ps)
-                        bulk_s2g(base + size_t(ps) * kRowBytes, smem + size_t(ps - d0) * kRowBytes,
-                                 uint32_t(pe - ps) * kRowBytes);
+                        for (int o = 0; o < pe - ps;) {
+                            const int nr = piece_rows(src + o, ps + o, pe - ps - o);
+                            bulk_s2g(row_ptr(ps + o), smem + size_t(ps + o - d0) * kRowBytes, uint32_t(nr) * kRowBytes);
+                            o += nr;
+                        }
                 }
                 bulk_commit();
             } else {
@@ -362,7 +378,7 @@ using namespace skipkv;
 
 static int compact_impl(const skipkv_shape* shape, void* K, void* V, const uint8_t* keep, const uint8_t* tok_keep,
                         int32_t* sent_off, int32_t* sent_id, int32_t* n_sent, int32_t* kv_len, int32_t* index_map,
-                        void* ws, void* stream) {
+                        void* ws, void* stream, const int32_t* block_table = nullptr, int max_pages = 0) {
     if (int rc = check_shape(shape)) return rc;
     if (!K || !V || !keep || !sent_off || !sent_id || !n_sent || !kv_len) return SKIPKV_ERR_INVALID_ARG;
     if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255)) return SKIPKV_ERR_WORKSPACE;
@@ -389,7 +405,7 @@ static int compact_impl(const skipkv_shape* shape, void* K, void* V, const uint8
     SKIPKV_CUDA(launch_dependent(compact_move_kernel, dim3(unsigned(num_sms() * 3)), dim3(kMoveThreads), kSegBytes, st,
                                  int(L.slabs), int(shape->n_kv_heads), int(shape->max_sent), shape->slab_off, shape->cap,
                                  static_cast<__nv_bfloat16*>(K), static_cast<__nv_bfloat16*>(V), index_map, hdr, nseg, loaded,
-                                 nruns, run_src, run_dst));
+                                 nruns, run_src, run_dst, block_table, max_pages));
     if (tok_keep && index_map)
         SKIPKV_CUDA(launch_dependent(compact_fill_index_kernel, dim3(L.slabs), dim3(64), 0, st, int(shape->n_kv_heads),
                                      shape->slab_off, shape->cap, tok_keep, index_map, static_cast<const int32_t*>(part)));
@@ -407,4 +423,12 @@ extern "C" int skipkv_compact_fill(const skipkv_shape* shape, void* K, void* V, 
                                    int32_t* kv_len, int32_t* index_map, void* ws, void* stream) {
     if (!tok_keep) return SKIPKV_ERR_INVALID_ARG;
     return compact_impl(shape, K, V, keep, tok_keep, sent_off, sent_id, n_sent, kv_len, index_map, ws, stream);
+}
+
+extern "C" int skipkv_compact_paged(const skipkv_shape* shape, void* K_pages, void* V_pages, const int32_t* block_table,
+                                    int32_t max_pages, const uint8_t* keep, int32_t* sent_off, int32_t* sent_id,
+                                    int32_t* n_sent, int32_t* kv_len, int32_t* index_map, void* ws, void* stream) {
+    if (!block_table || max_pages <= 0) return SKIPKV_ERR_INVALID_ARG;
+    return compact_impl(shape, K_pages, V_pages, keep, nullptr, sent_off, sent_id, n_sent, kv_len, index_map, ws, stream,
+                        block_table, max_pages);
 }

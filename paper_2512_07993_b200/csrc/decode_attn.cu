@@ -189,6 +189,11 @@ decode_attn_kernel(int batch, int Hq, int Hk, int n_slabs, const int64_t* slab_o
     // live rows of slab s; with a block table (paged cache) a slab cannot exceed its max_pages pages of kPageRows rows
     auto room = [&](int s) { return block_table ? min(cap[s / Hk], max_pages * kPageRows) : cap[s / Hk]; };
     auto old_len = [&](int s) { return min(max(kv_len[s], 0), room(s)); };     // rows before this launch
+    // cache row of token t of slab s (contiguous slabs, or through the block table)
+    auto phys_row = [&](int s, int t) {
+        return block_table ? size_t(max(block_table[size_t(s) * max_pages + t / kPageRows], 0)) * kPageRows + size_t(t % kPageRows)
+                           : slab_row0(slab_off, cap, Hk, s / Hk, s % Hk) + size_t(t);
+    };
     // rows streamed through the tile ring; with the fused step the row being appended is folded in separately
     auto live = [&](int s) { return old_len(s); };
     const int n = Hq / Hk;                     // heads per group
@@ -349,7 +354,7 @@ decode_attn_kernel(int batch, int Hq, int Hk, int n_slabs, const int64_t* slab_o
                     const int part = lane >> 4, c = lane & 15;
                     const uint4 val = (part ? step.v_new : step.k_new)[size_t(slab) * 16 + c];
                     reinterpret_cast<uint4*>(reinterpret_cast<uint8_t*>(wpart) + part * 2048)[c] = val;
-                    const size_t row = slab_row0(slab_off, cap, Hk, b, h) + size_t(old_len(slab));
+                    const size_t row = phys_row(slab, old_len(slab));
                     reinterpret_cast<uint4*>(const_cast<uint8_t*>(part ? V : K))[row * 16 + c] = val;
                 }
                 if (tid == kDecThreads - 33) { sm->step_n_sent = step.n_sent[slab]; sm->step_starts = step.new_sent[b]; }
@@ -519,7 +524,7 @@ decode_attn_kernel(int batch, int Hq, int Hk, int n_slabs, const int64_t* slab_o
                 for (int idx = tid; idx < n * kHeadDim; idx += kConsWarps * 32) o[idx] = vrow[idx % kHeadDim];
                 if (tid < 32) {
                     const int part = tid >> 4, c = tid & 15;
-                    const size_t row = slab_row0(slab_off, cap, Hk, b, h);
+                    const size_t row = phys_row(s, 0);
                     reinterpret_cast<uint4*>(const_cast<uint8_t*>(part ? V : K))[row * 16 + c] =
                         (part ? step.v_new : step.k_new)[size_t(s) * 16 + c];
                 }
@@ -607,6 +612,30 @@ extern "C" int skipkv_decode_step(const skipkv_shape* shape, const void* q, cons
     step.new_sent = new_sent; step.gen_id = gen_id; step.q_win = static_cast<uint4*>(q_win);
     step.window = shape->window; step.slot = slot; step.max_sent = shape->max_sent;
     return decode_impl(shape, q, K, V, kv_len_in, out, hidden, steer_vec, alpha, flag, nullptr, 0, step, ws, stream);
+}
+
+extern "C" int skipkv_decode_step_paged(const skipkv_shape* shape, const void* q, const void* k_new, const void* v_new,
+                                        void* K_pages, void* V_pages, const int32_t* block_table, int32_t max_pages,
+                                        const int32_t* kv_len_in, int32_t* kv_len_out, int32_t* sent_off, int32_t* sent_id,
+                                        int32_t* n_sent, const uint8_t* new_sent, const int32_t* gen_id, void* q_win,
+                                        int32_t slot, void* out, void* hidden, const void* steer_vec, const float* alpha,
+                                        const uint8_t* flag, void* ws, void* stream) {
+    if (!block_table || max_pages <= 0) return SKIPKV_ERR_INVALID_ARG;
+    if (!k_new || !v_new || !kv_len_in || !kv_len_out || kv_len_in == kv_len_out || !sent_off || !sent_id || !n_sent ||
+        !new_sent || !gen_id)
+        return SKIPKV_ERR_INVALID_ARG;
+    if (int rc = check_shape(shape)) return rc;
+    if (shape->max_sent <= 0) return SKIPKV_ERR_INVALID_ARG;
+    if (q_win && (slot < 0 || slot >= shape->window)) return SKIPKV_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(k_new) | reinterpret_cast<uintptr_t>(v_new) | reinterpret_cast<uintptr_t>(q_win)) & 15)
+        return SKIPKV_ERR_INVALID_ARG;
+    StepArgs step{};
+    step.k_new = static_cast<const uint4*>(k_new); step.v_new = static_cast<const uint4*>(v_new);
+    step.kv_len_out = kv_len_out; step.sent_off = sent_off; step.sent_id = sent_id; step.n_sent = n_sent;
+    step.new_sent = new_sent; step.gen_id = gen_id; step.q_win = static_cast<uint4*>(q_win);
+    step.window = shape->window; step.slot = slot; step.max_sent = shape->max_sent;
+    return decode_impl(shape, q, K_pages, V_pages, kv_len_in, out, hidden, steer_vec, alpha, flag, block_table, max_pages, step,
+                       ws, stream);
 }
 
 // ---------------------------------------------------------------------------------------------

@@ -74,6 +74,8 @@ struct SweepArgs {
     float* vsum;                        // [slabs][max_sent][128] sums of key rows
     uint32_t* status;
     const Header* hdr;
+    const int32_t* block_table;         // nullable: paged cache, tile j of slab s is page block_table[s * max_pages + j]
+    int max_pages;
 };
 
 // ---- sweep 1 epilogue: one accumulator (128 tokens) folded into the running (max, sum) of a row
@@ -181,7 +183,10 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_consta
     const int G = gridDim.x, cta = blockIdx.x;
     const int n_slabs = a.n_slabs, Hk = a.Hk, RB = a.RB;
     pdl_trigger();
-    auto live = [&](int s) { return min(max(a.kv_len[s], 0), a.cap[s / Hk]); };
+    auto live = [&](int s) {
+        const int room = a.block_table ? min(a.cap[s / Hk], a.max_pages * 128) : a.cap[s / Hk];
+        return min(max(a.kv_len[s], 0), room);
+    };
 
     if (tid == 0) {
         for (int s = 0; s < kSwMaxStages; ++s) {
@@ -253,8 +258,9 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_consta
                 }
                 if (lap > 0) ok = role_wait(&ctl->empty[stage], (lap - 1) & 1u, limit, &ctl->abort_flag, a.status);
                 if (!ok) break;
-                const long long row = (long long)slab_row0(a.slab_off, a.cap, Hk, slab / Hk, slab % Hk) +
-                                      (long long)(t - pref[slab]) * 128;
+                const long long row =
+                    a.block_table ? (long long)max(a.block_table[size_t(slab) * a.max_pages + (t - pref[slab])], 0) * 128
+                                  : (long long)slab_row0(a.slab_off, a.cap, Hk, slab / Hk, slab % Hk) + (long long)(t - pref[slab]) * 128;
                 uint8_t* dst = tiles + size_t(stage) * kOpBytes;
                 mbar_expect_tx(&ctl->full[stage], kOpBytes);
                 tma_load_2d(dst, &mapK, 0, int(row), &ctl->full[stage]);
@@ -362,7 +368,7 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_consta
                     while (pref[slab + 1] <= t) ++slab;
                     have = true;
                     N = live(slab);
-                    row0 = slab_row0(a.slab_off, a.cap, Hk, slab / Hk, slab % Hk);
+                    row0 = a.block_table ? size_t(slab) * a.max_pages * 128 : slab_row0(a.slab_off, a.cap, Hk, slab / Hk, slab % Hk);
                     // log-sum-exp of every query row of this slab from the sweep-1 records
                     const int fc = pref[slab] / per_cta, lc = (pref[slab + 1] - 1) / per_cta;
                     const float2* r0 = a.sc_part + size_t(fc + slab) * kSw1Groups * (size_t(RB) * 128);
@@ -830,7 +836,7 @@ using namespace skipkv;
 static int score_impl(const skipkv_shape* shape, const skipkv_params* params, const void* K, const void* q_win,
                       const int32_t* kv_len, const int32_t* sent_off, const int32_t* n_sent, float* tok_imp,
                       float* sent_imp, float* sent_red, float* sent_lam, float* sent_score, LamTable ext, void* ws,
-                      void* stream) {
+                      void* stream, const int32_t* block_table = nullptr, int max_pages = 0) {
     if (int rc = check_shape(shape)) return rc;
     if (!params || !K || !q_win || !kv_len || !sent_off || !n_sent || !sent_imp || !sent_red || !sent_lam || !sent_score)
         return SKIPKV_ERR_INVALID_ARG;
@@ -863,6 +869,7 @@ static int score_impl(const skipkv_shape* shape, const skipkv_params* params, co
     a.sc_part = reinterpret_cast<float2*>(w + L.sc_part);
     a.tok_imp_user = tok_imp; a.tok_imp_ws = sc_tok; a.vsum = vsum; a.status = status;
     a.hdr = reinterpret_cast<const Header*>(w + L.header);
+    a.block_table = block_table; a.max_pages = max_pages;
     const size_t max_smem = 227 * 1024;
     const size_t fixed1 = 1024 + size_t(a.RB) * kOpBytes + sizeof(SweepCtl) + size_t(L.slabs + 1) * 4;
     if (fixed1 + kOpBytes > max_smem) return SKIPKV_ERR_UNSUPPORTED;
@@ -935,4 +942,15 @@ extern "C" int skipkv_score_table(const skipkv_shape* shape, const skipkv_params
     if (int rc = check_shape(shape)) return rc;
     return score_impl(shape, params, K, q_win, kv_len, sent_off, n_sent, tok_imp, sent_imp, sent_red, sent_lam,
                       sent_score, LamTable{lam_table, sent_id, table_len, shape->n_kv_heads}, ws, stream);
+}
+
+extern "C" int skipkv_score_paged(const skipkv_shape* shape, const skipkv_params* params, const void* K_pages,
+                                  const int32_t* block_table, int32_t max_pages, const void* q_win, const int32_t* kv_len,
+                                  const int32_t* sent_off, const int32_t* n_sent, float* tok_imp, float* sent_imp,
+                                  float* sent_red, float* sent_lam, float* sent_score, void* ws, void* stream) {
+    if (!block_table || max_pages <= 0) return SKIPKV_ERR_INVALID_ARG;
+    if (int rc = check_shape(shape)) return rc;
+    if (int64_t(max_pages) * 128 > int64_t(shape->max_cap) + 127) return SKIPKV_ERR_INVALID_ARG;   // the workspace is sized by max_cap
+    return score_impl(shape, params, K_pages, q_win, kv_len, sent_off, n_sent, tok_imp, sent_imp, sent_red, sent_lam,
+                      sent_score, LamTable{nullptr, nullptr, 0, 1}, ws, stream, block_table, max_pages);
 }
