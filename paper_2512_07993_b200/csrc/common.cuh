@@ -197,6 +197,8 @@ __device__ __forceinline__ void bulk_wait_read_all() {
     asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
 }
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
+// The same for shared memory only (generic writes to shared memory that the tensor core or a bulk copy reads next).
+__device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 // The wait limit a workspace carries (skipkv_set_wait_limit); 0 stands for the default.
 __device__ __forceinline__ uint32_t load_wait_limit(const Header* hdr) {

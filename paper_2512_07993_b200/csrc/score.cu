@@ -4,7 +4,8 @@
 //             (tensor cores: logits = Q_group x K_tile^T, one thread per query row)
 //   sweep 2   tok_imp[t] = (1/alpha) sum_w max_q 2^(s_q[w][t] - lse_q[w])   (max before exp: exp is monotone)
 //             (tensor cores: logits = K_tile x Q_group^T, one thread per token), and in the same pass
-//             the per-sentence sums of the key rows, taken from the tile already in shared memory
+//             the per-sentence sums of the key rows as a second product on the tile already in shared
+//             memory: K_tile^T x (0/1 matrix token -> sentence slot)
 //   pool      per sentence: mean tok_imp, mean key, normalisation, split into bf16 high and low parts
 //   gram x2   pairwise cosine G on the tensor cores (three bf16 products: hi.hi + hi.lo + lo.hi);
 //             pass 1: Z_i = sum_{j!=i} e^{G_ij} and lam_i = max_{j>i} G_ij;
@@ -16,7 +17,8 @@
 // Both sweeps are persistent, warp-specialised kernels, one CTA per SM: a TMA warp streams
 // 128-token key tiles (and the group's query block) into shared memory, one thread issues
 // tcgen05.mma into a ring of four tensor-memory accumulators, several warpgroups of epilogue warps
-// take the tiles round-robin, and (sweep 2) one more warpgroup pools the key rows.  Work is the list of
+// take the tiles round-robin, and (sweep 2) one more warpgroup builds the 0/1 matrices of the pooling product,
+// issues it and drains the pooled sums.  Work is the list of
 // 128-token tiles over all slabs cut into equal contiguous ranges, so ragged slabs balance.
 //
 // Query rows of a group are staged as blocks of WB = floor(128/n) window positions x n heads
@@ -34,9 +36,14 @@ constexpr int kMaxRB = 4;               // query blocks per group
 constexpr int kSwMaxStages = 6;
 constexpr int kSw1Groups = 4;           // epilogue warpgroups of sweep 1
 constexpr int kSw2Groups = 2;           // epilogue warpgroups of sweep 2
-constexpr int kPoolWarps = 8;           // pooling warps of sweep 2: warp p sums rows 32 (p & 3) .. +31 of the tiles of parity p >> 2
+constexpr int kSw2Bufs = 3;             // sweep 2: accumulators of the logits (the columns after them hold the pooled sums)
+constexpr int kPoolWarps = 4;           // sweep 2: the warpgroup that writes the indicator matrices and drains the pooled sums
+constexpr int kIndRing = 2;             // indicator matrices (and pooled-sum accumulators) in flight
+constexpr int kIndSlots = 16;           // sentence slots of one indicator matrix
+constexpr int kIndBytes = kIndSlots * 128 * 2;   // [16 slots][128 tokens] bf16 as two 64-token halves, 128-byte swizzle
+constexpr uint32_t kPoolCol = kSw2Bufs * 128;    // tensor-memory column of the first pooled-sum accumulator (16 columns each)
 constexpr int kSw1Threads = (2 + 4 * kSw1Groups) * 32;        // TMA warp, MMA warp, epilogue warps
-constexpr int kSw2Threads = (2 + 4 * kSw2Groups + kPoolWarps) * 32;
+constexpr int kSw2Threads = (2 + 4 * kSw2Groups + kPoolWarps + 1) * 32;   // + the thread that issues the pooling products
 constexpr float kLog2e = 1.4426950408889634f;
 
 __device__ __forceinline__ float ex2f(float x) {
@@ -54,7 +61,10 @@ struct SweepCtl {                       // barriers and small shared state, afte
     uint64_t tfull[4][4], tempty[kAccBufs];
     uint32_t tmem_base;
     int abort_flag;
-    int landed;                         // sweep 2: tiles whose copy has completed (a monotone count for the pooling warps)
+    // sweep 2, ring of indicator matrices: written by the four pooling warps -> multiplied by the MMA thread -> drained by
+    // the pooling warps
+    uint64_t ifull[kIndRing], pfull[kIndRing];
+    int ind_more[kIndRing];             // "the tile has another matrix after this one"
     uint32_t wsum[32];
     alignas(16) float neg_lse[kSw2Groups][kMaxRB * 128];   // sweep 2: one copy per epilogue warpgroup (read as float4)
 };
@@ -62,7 +72,6 @@ static_assert(offsetof(SweepCtl, neg_lse) % 16 == 0, "neg_lse is read with 16-by
 
 struct SweepArgs {
     int Hq, Hk, window, n_slabs, max_cap, max_sent, RB, WB, stages;
-    int so_smem;                        // sweep 2: sentence offsets and per-tile first sentences are staged in shared memory
     const int64_t* slab_off;
     const int32_t* cap;
     const int32_t* kv_len;
@@ -166,6 +175,50 @@ __device__ __forceinline__ float imp_fold(uint32_t taddr, const float* neg_lse, 
     return total;
 }
 
+// ---- sweep 2: pooled key sums on the tensor cores
+// Pooling product of one staged tile: D[128 channels x 16 slots] = K_tile^T x Ind^T.  A = the tile as the TMA load
+// wrote it ([token][channel], two 64-channel halves, 128-byte swizzle) read as an MN-major operand: 64 channels x 8
+// tokens per swizzle atom, atoms 1024 bytes apart along the tokens and a half (16 KB) apart along the channels.
+// B = the indicator matrix [slot][token], K-major like every other operand here.
+constexpr uint32_t kIdescPool = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | ((uint32_t(kIndSlots) >> 3) << 17) |
+                                ((128u >> 4) << 24);
+__device__ __forceinline__ void umma_pool(uint32_t tmem_d, uint32_t tile_smem, uint32_t ind_smem) {
+#pragma unroll
+    for (int ks = 0; ks < 8; ++ks) {                     // 16 tokens per step
+        const uint32_t a_addr = tile_smem + ks * 2048;
+        const uint64_t da = uint64_t((a_addr >> 4) & 0x3fffu) | (uint64_t(kOpHalfBytes >> 4) << 16) |
+                            (uint64_t(1024 >> 4) << 32) | (uint64_t(1) << 46) | (uint64_t(2) << 61);
+        const uint64_t db = umma_desc_sw128(ind_smem + (ks >> 2) * (kIndBytes / 2) + (ks & 3) * 32);
+        umma_bf16(tmem_d, da, db, kIdescPool, ks ? 1u : 0u);
+    }
+}
+// 16 consecutive fp32 columns of this thread's tensor-memory lane.
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
+    uint32_t r[16];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];\n\t"
+        "tcgen05.wait::ld.sync.aligned;"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr)
+        : "memory");
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+// One 16-byte piece of an indicator matrix: tokens 8c .. 8c + 7 of slot row j; ones (bf16 1.0) for the tokens
+// [lo, hi), zeros elsewhere.
+__device__ __forceinline__ void indicator_piece(uint8_t* ind, int j, int c, int lo, int hi) {
+    const int b0 = min(max(lo - 8 * c, 0), 8), b1 = min(max(hi - 8 * c, 0), 8);
+    const uint32_t m8 = b1 > b0 ? (((1u << b1) - 1u) & ~((1u << b0) - 1u)) : 0u;
+    uint4 val;
+    val.x = (m8 & 1u) * 0x3F80u + ((m8 >> 1) & 1u) * 0x3F800000u;
+    val.y = ((m8 >> 2) & 1u) * 0x3F80u + ((m8 >> 3) & 1u) * 0x3F800000u;
+    val.z = ((m8 >> 4) & 1u) * 0x3F80u + ((m8 >> 5) & 1u) * 0x3F800000u;
+    val.w = ((m8 >> 6) & 1u) * 0x3F80u + ((m8 >> 7) & 1u) * 0x3F800000u;
+    *reinterpret_cast<uint4*>(ind + (c >> 3) * (kIndBytes / 2) + j * 128 + (((c & 7) ^ (j & 7)) << 4)) = val;
+}
+
 template <int kSweep, int kN>
 __global__ void __launch_bounds__(kSweep == 1 ? kSw1Threads : kSw2Threads, 1)
 score_sweep_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapQ,
@@ -176,7 +229,8 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_consta
     const uint32_t raw = smem_u32(sweep_smem_raw);
     uint8_t* tiles = sweep_smem_raw + (((raw + 1023u) & ~1023u) - raw);          // 1024-byte aligned
     uint8_t* qbuf = tiles + size_t(a.stages) * kOpBytes;
-    SweepCtl* ctl = reinterpret_cast<SweepCtl*>(qbuf + size_t(a.RB) * kOpBytes);
+    uint8_t* indb = qbuf + size_t(a.RB) * kOpBytes;                              // sweep 2: the indicator matrices
+    SweepCtl* ctl = reinterpret_cast<SweepCtl*>(indb + (kSweep == 2 ? kIndRing * kIndBytes : 0));
     int* pref = reinterpret_cast<int*>(ctl + 1);                                 // [n_slabs + 1] tile prefix
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -191,15 +245,15 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_consta
     if (tid == 0) {
         for (int s = 0; s < kSwMaxStages; ++s) {
             mbar_init(&ctl->full[s], 1);
-            mbar_init(&ctl->empty[s], kSweep == 1 ? 1 : 5);      // MMA commit (+ the tile's four pooling warps)
+            mbar_init(&ctl->empty[s], kSweep == 1 ? 1 : 2);      // commit of the logits (+ commit of the tile's last pooling product)
         }
         mbar_init(&ctl->qfull, 1);
         mbar_init(&ctl->qempty, 1);
         for (int b = 0; b < kAccBufs; ++b) mbar_init(&ctl->tempty[b], 4);
         for (int g = 0; g < 4; ++g)
             for (int j = 0; j < 4; ++j) mbar_init(&ctl->tfull[g][j], 1);
+        for (int i = 0; i < kIndRing; ++i) { mbar_init(&ctl->ifull[i], kPoolWarps); mbar_init(&ctl->pfull[i], 1); }
         ctl->abort_flag = 0;
-        ctl->landed = 0;
         mbar_fence_init();
         tmap_prefetch(&mapK);
         tmap_prefetch(&mapQ);
@@ -239,12 +293,17 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_consta
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0 && ntl > 0) {
-            int slab = slab0, stage = 0, issued = 0;
+            // what depends on the slab only is kept in registers: between "stage free" and the next copy's issue nothing
+            // waits on shared or global memory
+            int slab = slab0, stage = 0, issued = 0, slab_begin = 0, slab_end = 0;
+            long long row0 = 0;
             uint32_t lap = 0, qlap = 0;
             bool ok = true;
             for (int t = t_begin; t < t_end && ok; ++t) {
-                if (t == t_begin || pref[slab + 1] <= t) {
+                if (t == t_begin || slab_end <= t) {
                     while (pref[slab + 1] <= t) ++slab;
+                    slab_begin = pref[slab]; slab_end = pref[slab + 1];
+                    row0 = a.block_table ? 0 : (long long)slab_row0(a.slab_off, a.cap, Hk, slab / Hk, slab % Hk);
                     if (qlap > 0) ok = role_wait(&ctl->qempty, (qlap - 1) & 1u, limit, &ctl->abort_flag, a.status);
                     if (!ok) break;
                     const int b = slab / Hk, h = slab % Hk;
@@ -256,11 +315,11 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_consta
                     }
                     ++qlap;
                 }
+                const long long row =
+                    a.block_table ? (long long)max(a.block_table[size_t(slab) * a.max_pages + (t - slab_begin)], 0) * 128
+                                  : row0 + (long long)(t - slab_begin) * 128;
                 if (lap > 0) ok = role_wait(&ctl->empty[stage], (lap - 1) & 1u, limit, &ctl->abort_flag, a.status);
                 if (!ok) break;
-                const long long row =
-                    a.block_table ? (long long)max(a.block_table[size_t(slab) * a.max_pages + (t - pref[slab])], 0) * 128
-                                  : (long long)slab_row0(a.slab_off, a.cap, Hk, slab / Hk, slab % Hk) + (long long)(t - pref[slab]) * 128;
                 uint8_t* dst = tiles + size_t(stage) * kOpBytes;
                 mbar_expect_tx(&ctl->full[stage], kOpBytes);
                 tma_load_2d(dst, &mapK, 0, int(row), &ctl->full[stage]);
@@ -278,25 +337,23 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_consta
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0 && ntl > 0) {
-            int slab = slab0, stage = 0, it = 0;
+            int slab = slab0, stage = 0, it = 0, slab_end = 0;
             uint32_t lap = 0, qlap = 0;
             bool ok = true;
             for (int t = t_begin; t < t_end && ok; ++t) {
-                if (t == t_begin || pref[slab + 1] <= t) {
+                if (t == t_begin || slab_end <= t) {
                     while (pref[slab + 1] <= t) ++slab;
+                    slab_end = pref[slab + 1];
                     ok = role_wait(&ctl->qfull, qlap & 1u, limit, &ctl->abort_flag, a.status);
                     if (!ok) break;
                     ++qlap;
                 }
                 ok = role_wait(&ctl->full[stage], lap & 1u, limit, &ctl->abort_flag, a.status);
                 if (!ok) break;
-                if (kSweep == 2) {                       // pooling warps skip tiles, so they follow a count, not barrier phases
-                    __threadfence_block();
-                    *reinterpret_cast<volatile int*>(&ctl->landed) = t - t_begin + 1;
-                }
                 const uint32_t k_smem = smem_u32(tiles + size_t(stage) * kOpBytes);
                 for (int k = 0; k < RB && ok; ++k, ++it) {
-                    const int buf = it & (kAccBufs - 1), use = it / kAccBufs;
+                    constexpr int kBufs = kSweep == 1 ? kAccBufs : kSw2Bufs;
+                    const int buf = it % kBufs, use = it / kBufs;
                     if (use > 0) ok = role_wait(&ctl->tempty[buf], uint32_t(use - 1) & 1u, limit, &ctl->abort_flag, a.status);
                     if (!ok) break;
                     tc_fence_after();
@@ -308,8 +365,8 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_consta
                         umma_commit(&ctl->tfull[ti % kGroups][gj & 3]);
                     }
                 }
+                if (t + 1 == t_end || slab_end <= t + 1) umma_commit(&ctl->qempty);
                 umma_commit(&ctl->empty[stage]);
-                if (t + 1 == t_end || pref[slab + 1] <= t + 1) umma_commit(&ctl->qempty);
                 if (++stage == a.stages) { stage = 0; ++lap; }
             }
         }
@@ -390,7 +447,7 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_consta
 #pragma unroll
                 for (int k = 0; k < kMaxRB; ++k) {
                     if (k < RB && ok) {
-                        const int it = tl * RB + k, buf = it & (kAccBufs - 1);
+                        const int it = tl * RB + k, buf = it % kSw2Bufs;
                         const int gj = (tl / kGroups) * RB + k;
                         ok = role_wait(&ctl->tfull[g][gj & 3], uint32_t(gj >> 2) & 1u, limit, &ctl->abort_flag, a.status);
                         ok = __all_sync(0xffffffffu, ok);
@@ -412,118 +469,159 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_consta
                 }
             }
         }
-    } else if (kSweep == 2) {
-        // ------------------------------------------------------------------ pooling warps: per-sentence sums of key rows
-        // Loads from shared memory wait several hundred cycles here (the tensor core streams its operands from the
-        // same memory), and a tile's stage is held until its pooling is done, so the work is arranged for few
-        // dependent steps and a short hold: four warps share a tile (32 rows each), two such groups alternate over
-        // the tiles; the sentence of a 32-row block's first token comes from a table built once per slab; the starts
-        // of the following sentences are fetched in one access; a warp's rows are loaded sixteen at a time.  A lane
-        // owns 4 channels (8 bytes) of every row.
-        const int pw = warp - (2 + 4 * kGroups);
-        const int ptid = tid - (2 + 4 * kGroups) * 32;                 // thread index among the pooling warps
-        const int half = lane >> 4, chunk = (lane & 15) >> 1, sub = (lane & 1) * 8;
-        const int ch0 = half * 64 + (lane & 15) * 4;                   // first channel of this lane
-        int32_t* so_stage = reinterpret_cast<int32_t*>(pref + n_slabs + 1);       // [max_sent + 1]
-        int32_t* tfirst = so_stage + (a.max_sent + 1);                            // [tiles of the slab]
-        int slab = slab0, S = 0, N = 0;
+    } else if (kSweep == 2 && warp < 2 + 4 * kGroups + kPoolWarps) {
+        // ------------------------------------------------------------------ per-sentence sums of the key rows
+        // The sums are a product on the tensor cores: (tile^T: channel x token) x (indicator: token x sentence slot).
+        // Slot 0 of a tile's first matrix is a sentence that starts at or before the tile's first token; a tile that
+        // touches more than 16 sentences (empty ones count) gets further matrices.  Each of the four warps writes a
+        // quarter of the matrix and arrives; one thread of a fifth warp issues the product, and while it runs every warp
+        // adds the previous product (a thread owns one channel) to the sums in global memory.
+        // Every warp keeps, one entry per lane, a window of the slab's sentence offsets starting at entry `base`
+        // (entries past the table read as "never starts"), refilled from global memory when a tile needs entries
+        // beyond it: loads from shared memory wait several hundred cycles here (the tensor core streams its operands
+        // from it), so the per-tile work touches shared memory only to write the matrix.
+        constexpr int kNever = 0x7fffffff;
+        const int gw = warp - (2 + 4 * kGroups);                // warp of the group: slots 4 gw .. 4 gw + 3 of a matrix
+        const int gtid = tid - (2 + 4 * kGroups) * 32;
+        const int quarter = warp & 3;                           // tensor-memory lanes this warp may read
+        const int ch = quarter * 32 + lane;
+        const uint32_t lane_addr = tmem_base + (uint32_t(quarter * 32) << 16) + kPoolCol;
+        int slab = slab0, S = 0, N = 0, ic = 0, first = 0, base = 0, w = kNever;
         const int32_t* so = a.sent_off;
         bool ok = true, have = false;
-        for (int tl = 0; tl < ntl; ++tl) {
-            const int t = t_begin + tl, stage = tl % a.stages;
-            if (!have || pref[slab + 1] <= t) {
-                // new slab (all pooling warps get here at the same tile): stage its sentence offsets and the
-                // sentence of every tile's first token; the first barrier ends the reads of the old tables
+        // the product still to be drained: its accumulator, sentence of slot 0, slots that hold tokens
+        bool pend = false;
+        int p_slab = 0, p_first = 0;
+        uint32_t p_held = 0;
+        auto refill = [&](int b) { base = b; w = (b + lane <= S) ? so[b + lane] : kNever; };
+        auto drain = [&]() {
+            const int is = (ic - 1) & (kIndRing - 1);
+            ok = role_wait(&ctl->pfull[is], uint32_t((ic - 1) / kIndRing) & 1u, limit, &ctl->abort_flag, a.status);
+            ok = __all_sync(0xffffffffu, ok);
+            if (ok) {
+                tc_fence_after();
+                float v[kIndSlots];
+                tmem_ld16(lane_addr + uint32_t(is) * kIndSlots, v);
+                tc_fence_before();
+                float* dst = a.vsum + (size_t(p_slab) * a.max_sent + p_first) * kHeadDim + ch;
+#pragma unroll
+                for (int j = 0; j < kIndSlots; ++j)
+                    if (p_held & (1u << j)) atomicAdd(dst + size_t(j) * kHeadDim, v[j]);
+            }
+            pend = false;
+        };
+        for (int tl = 0; tl < ntl && ok; ++tl) {
+            const int t = t_begin + tl;
+            const bool fresh = !have || pref[slab + 1] <= t;
+            int w0 = kNever;
+            if (fresh) {
                 while (pref[slab + 1] <= t) ++slab;
                 have = true;
-                S = min(max(a.n_sent[slab], 0), a.max_sent);
                 so = a.sent_off + size_t(slab) * (a.max_sent + 1);
+                w0 = lane <= a.max_sent ? so[lane] : kNever;        // issued together with the loads of the lengths
+                S = min(max(a.n_sent[slab], 0), a.max_sent);
                 N = live(slab);
-                if (a.so_smem) {
-                    named_bar_sync(8, kPoolWarps * 32);
-                    for (int i = ptid; i <= S; i += kPoolWarps * 32) so_stage[i] = so[i];
-                    named_bar_sync(8, kPoolWarps * 32);
-                    so = so_stage;
-                    const int nt = (N + 31) >> 5;                   // 32-row blocks of the slab
-                    for (int j = ptid; j < nt; j += kPoolWarps * 32) {
-                        int lo = 0, hi = max(S - 1, 0);
-                        while (lo < hi) {
-                            const int mid = (lo + hi + 1) >> 1;
-                            if (so[mid] <= j * 32) lo = mid; else hi = mid - 1;
-                        }
-                        tfirst[j] = lo;
-                    }
-                    named_bar_sync(8, kPoolWarps * 32);
+            }
+            const int tok0 = (t - pref[slab]) * 128, valid = min(128, N - tok0);
+            const int stage = tl % a.stages;
+            if (fresh) {
+                // the last sentence that starts at or before the first token: at the head of a slab it is among the first
+                // entries (already loaded) unless the slab opens with 32 empty sentences
+                base = 0;
+                w = lane <= S ? w0 : kNever;
+                const int n_le = __popc(__ballot_sync(0xffffffffu, lane < S && w <= tok0));
+                first = max(n_le - 1, 0);
+            }
+            if (fresh && (tok0 > 0 || first >= 31)) {
+                // elsewhere: a 32-way search, one probe per lane
+                int lo = 0, len = S;
+                while (len > 32) {
+                    const int stride = (len + 31) >> 5;
+                    const int pidx = lo + lane * stride;
+                    const bool le = pidx < lo + len && so[pidx] <= tok0;
+                    const int adv = max(__popc(__ballot_sync(0xffffffffu, le)) - 1, 0) * stride;
+                    len = min(stride, len - adv);
+                    lo += adv;
+                }
+                const bool le = lane < len && so[lo + lane] <= tok0;
+                first = lo + max(__popc(__ballot_sync(0xffffffffu, le)) - 1, 0);
+                refill(first);
+            }
+            // every warp follows every tile's arrival (in order, so it sees each phase of the stage's barrier)
+            ok = role_wait(&ctl->full[stage], uint32_t(tl / a.stages) & 1u, limit, &ctl->abort_flag, a.status);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            if (valid < 128) {
+                // a zero in the indicator does not silence a NaN or an infinity in a dead row: clear the rows past the
+                // slab's end in the staged tile (the logits of those rows are never read)
+                uint8_t* tile = tiles + size_t(stage) * kOpBytes;
+                for (int u = valid * 8 + gtid; u < 128 * 8; u += kPoolWarps * 32) {
+                    *reinterpret_cast<uint4*>(tile + u * 16) = make_uint4(0u, 0u, 0u, 0u);
+                    *reinterpret_cast<uint4*>(tile + kOpHalfBytes + u * 16) = make_uint4(0u, 0u, 0u, 0u);
                 }
             }
-            if ((tl & 1) != (pw >> 2)) continue;                // the other group's tile
-            if (ok) {                                           // wait (bounded) until the tile's copy has landed
-                uint32_t spins = 0;
-                while (*reinterpret_cast<volatile int*>(&ctl->landed) <= tl) {
-                    if (*reinterpret_cast<volatile int*>(&ctl->abort_flag) || ++spins > limit) { ok = false; break; }
-                    __nanosleep(64);
+            int more = 0;
+            do {
+                const int is = ic & (kIndRing - 1);
+                if (first < base || first + kIndSlots > base + 31) refill(first);
+                const int d = first - base;                         // window position of slot 0's sentence
+                // tile-relative start of every window entry, clamped to the tile; slot j holds [cl(d + j), cl(d + j + 1))
+                const int cl = min(max(min(w, tok0 + valid) - tok0, 0), valid);
+                const int cl_next = __shfl_down_sync(0xffffffffu, cl, 1);
+                const uint32_t holds = __ballot_sync(0xffffffffu, base + lane < S && lane < 31 && cl_next > cl);
+                const uint32_t held = (holds >> d) & 0xffffu;       // bit j: slot j holds tokens
+                const int s_next = __shfl_sync(0xffffffffu, w, d + kIndSlots);   // start of the sentence after slot 15
+                more = (first + kIndSlots < S && s_next < tok0 + valid) ? 1 : 0;
+                // sentences after slot 0 that start at or before the next tile's first token: the last of them is a
+                // valid slot 0 there
+                const bool in_next = lane > d && lane <= d + kIndSlots && base + lane < S && w <= tok0 + 128;
+                const int step = __popc(__ballot_sync(0xffffffffu, in_next));
+                {
+                    const int j = 4 * gw + (lane >> 3);             // this thread's slot row and its two pieces
+                    const int lo = __shfl_sync(0xffffffffu, cl, d + j), hi = __shfl_sync(0xffffffffu, cl, d + j + 1);
+                    const bool is_sent = (held >> j) & 1u;
+                    indicator_piece(indb + size_t(is) * kIndBytes, j, (lane & 7) * 2, is_sent ? lo : 0, is_sent ? hi : 0);
+                    indicator_piece(indb + size_t(is) * kIndBytes, j, (lane & 7) * 2 + 1, is_sent ? lo : 0, is_sent ? hi : 0);
                 }
-                ok = __all_sync(0xffffffffu, ok);
-                if (!ok && lane == 0) {
-                    atomicOr(a.status, SKIPKV_STATUS_COPY_TIMEOUT);
-                    *reinterpret_cast<volatile int*>(&ctl->abort_flag) = 1;
+                fence_proxy_async_smem();                           // the matrix (and cleared rows) are read by the tensor core
+                tc_fence_before();                                  // and this warp's reads of the accumulator came first
+                __syncwarp();
+                if (lane == 0) {
+                    if (gw == 0) ctl->ind_more[is] = more;
+                    mbar_arrive(&ctl->ifull[is]);
                 }
-                __threadfence_block();
+                if (pend) drain();                                  // the previous product, while this one runs
+                if (!ok) break;
+                pend = true; p_slab = slab; p_first = first; p_held = held;
+                ++ic;
+                first = more ? first + kIndSlots : first + step;
+            } while (more);
+        }
+        if (pend && ok) drain();
+    } else if (kSweep == 2) {
+        // ------------------------------------------------------------------ issuer of the pooling products
+        // (its own thread: an issue blocks for the length of the product, and every look at shared memory costs the
+        // thread that issues the logits a few hundred cycles)
+        if (lane == 0 && ntl > 0) {
+            const uint32_t indb_u32 = smem_u32(indb);
+            bool ok = true;
+            int pc = 0;
+            for (int tl = 0; tl < ntl && ok; ++tl) {
+                const int stage = tl % a.stages;
+                int more = 0;
+                do {
+                    const int is = pc & (kIndRing - 1);
+                    ok = role_wait(&ctl->ifull[is], uint32_t(pc / kIndRing) & 1u, limit, &ctl->abort_flag, a.status);
+                    if (!ok) break;
+                    more = *reinterpret_cast<volatile int*>(&ctl->ind_more[is]);
+                    tc_fence_after();
+                    umma_pool(tmem_base + kPoolCol + uint32_t(is) * kIndSlots, smem_u32(tiles + size_t(stage) * kOpBytes),
+                              indb_u32 + uint32_t(is) * kIndBytes);
+                    umma_commit(&ctl->pfull[is]);
+                    ++pc;
+                } while (more);
+                if (ok) umma_commit(&ctl->empty[stage]);
             }
-            if (!ok) continue;
-            const int row0 = (pw & 3) * 32;                     // this warp's rows of the tile: [row0, row0 + 32)
-            const int tok0 = (t - pref[slab]) * 128 + row0;
-            const int nrows = min(32, N - tok0);
-            if (S > 0 && nrows > 0) {
-                int cur;
-                if (a.so_smem) {
-                    cur = tfirst[tok0 >> 5];
-                } else {
-                    int lo = 0, hi = S - 1;
-                    while (lo < hi) {
-                        const int mid = (lo + hi + 1) >> 1;
-                        if (so[mid] <= tok0) lo = mid; else hi = mid - 1;
-                    }
-                    cur = lo;
-                }
-                // tile-relative starts of the next 32 sentences, one per lane (refilled if a tile has more)
-                int base = cur + 1;
-                int my = (base + lane < S) ? so[base + lane] - tok0 : 0x7fffffff;
-                const uint8_t* colbase = tiles + size_t(stage) * kOpBytes + half * kOpHalfBytes + row0 * 128 + sub;
-                float* dst = a.vsum + size_t(slab) * a.max_sent * kHeadDim + ch0;
-                int r = 0;
-                while (r < nrows) {
-                    // piece [r, e): rows of sentence `cur`
-                    int e = nrows;
-                    if (cur + 1 < S) {
-                        if (cur + 1 - base >= 32) { base = cur + 1; my = (base + lane < S) ? so[base + lane] - tok0 : 0x7fffffff; }
-                        e = min(e, __shfl_sync(0xffffffffu, my, cur + 1 - base));
-                    }
-                    if (e > r) {
-                        float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-#pragma unroll 1
-                        for (int rb = r; rb < e; rb += 16) {    // sixteen rows in flight; rows past the piece load as zero
-                            uint2 u[16];
-#pragma unroll
-                            for (int i = 0; i < 16; ++i) {
-                                const int rr = rb + i;
-                                u[i] = (rr < e) ? *reinterpret_cast<const uint2*>(colbase + rr * 128 + ((chunk ^ (rr & 7)) << 4))
-                                                : make_uint2(0u, 0u);
-                            }
-#pragma unroll
-                            for (int i = 0; i < 16; ++i) {
-                                a0 += bf16lo(u[i].x); a1 += bf16hi(u[i].x);
-                                a2 += bf16lo(u[i].y); a3 += bf16hi(u[i].y);
-                            }
-                        }
-                        atomicAdd(reinterpret_cast<float4*>(dst + size_t(cur) * kHeadDim), make_float4(a0, a1, a2, a3));
-                        r = e;
-                    }
-                    if (r < nrows) ++cur;                       // the piece ended on a sentence boundary
-                }
-            }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&ctl->empty[stage]);
         }
     }
     tc_fence_before();
@@ -874,14 +972,11 @@ static int score_impl(const skipkv_shape* shape, const skipkv_params* params, co
     const size_t fixed1 = 1024 + size_t(a.RB) * kOpBytes + sizeof(SweepCtl) + size_t(L.slabs + 1) * 4;
     if (fixed1 + kOpBytes > max_smem) return SKIPKV_ERR_UNSUPPORTED;
     SweepArgs a1 = a, a2 = a;
-    a1.so_smem = 0;
     a1.stages = int((max_smem - fixed1) / kOpBytes);
     if (a1.stages > kSwMaxStages) a1.stages = kSwMaxStages;
-    // sweep 2 also stages the current slab's sentence offsets and one sentence index per 32 rows of the slab, when
-    // that leaves at least two tile stages (otherwise its pooling warps read the table from global memory)
-    const size_t tab_bytes = (size_t(shape->max_sent) + 1 + size_t((shape->max_cap + 31) / 32)) * 4;
-    a2.so_smem = (fixed1 + tab_bytes + 2 * kOpBytes <= max_smem) ? 1 : 0;
-    const size_t fixed2 = fixed1 + (a2.so_smem ? tab_bytes : 0);
+    // sweep 2 also holds the indicator matrices of its pooling product
+    const size_t fixed2 = fixed1 + size_t(kIndRing) * kIndBytes;
+    if (fixed2 + kOpBytes > max_smem) return SKIPKV_ERR_UNSUPPORTED;
     a2.stages = int((max_smem - fixed2) / kOpBytes);
     if (a2.stages > kSwMaxStages) a2.stages = kSwMaxStages;
     const size_t smem1 = fixed1 + size_t(a1.stages) * kOpBytes, smem2 = fixed2 + size_t(a2.stages) * kOpBytes;
