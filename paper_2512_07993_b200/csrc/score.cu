@@ -38,7 +38,7 @@ constexpr int kSw1Groups = 4;           // epilogue warpgroups of sweep 1
 constexpr int kSw2Groups = 2;           // epilogue warpgroups of sweep 2
 constexpr int kSw2Bufs = 3;             // sweep 2: accumulators of the logits (the columns after them hold the pooled sums)
 constexpr int kPoolWarps = 4;           // sweep 2: the warpgroup that writes the indicator matrices and drains the pooled sums
-constexpr int kIndRing = 2;             // indicator matrices (and pooled-sum accumulators) in flight
+constexpr int kIndRing = 2;             // indicator matrices in flight (the pooled sums have two accumulators of their own)
 constexpr int kIndSlots = 16;           // sentence slots of one indicator matrix
 constexpr int kIndBytes = kIndSlots * 128 * 2;   // [16 slots][128 tokens] bf16 as two 64-token halves, 128-byte swizzle
 constexpr uint32_t kPoolCol = kSw2Bufs * 128;    // tensor-memory column of the first pooled-sum accumulator (16 columns each)
@@ -63,8 +63,9 @@ struct SweepCtl {                       // barriers and small shared state, afte
     int abort_flag;
     // sweep 2, ring of indicator matrices: written by the four pooling warps -> multiplied by the MMA thread -> drained by
     // the pooling warps
-    uint64_t ifull[kIndRing], pfull[kIndRing];
-    int ind_more[kIndRing];             // "the tile has another matrix after this one"
+    uint64_t ifull[kIndRing], iempty[kIndRing];
+    uint64_t pfull[2];                  // the last product of a run of tiles into accumulator i has completed
+    int ind_flags[kIndRing];            // 1: the tile has another matrix after this one, 2: joins the open run, 4: closes a run
     uint32_t wsum[32];
     alignas(16) float neg_lse[kSw2Groups][kMaxRB * 128];   // sweep 2: one copy per epilogue warpgroup (read as float4)
 };
@@ -182,14 +183,14 @@ __device__ __forceinline__ float imp_fold(uint32_t taddr, const float* neg_lse, 
 // B = the indicator matrix [slot][token], K-major like every other operand here.
 constexpr uint32_t kIdescPool = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | ((uint32_t(kIndSlots) >> 3) << 17) |
                                 ((128u >> 4) << 24);
-__device__ __forceinline__ void umma_pool(uint32_t tmem_d, uint32_t tile_smem, uint32_t ind_smem) {
+__device__ __forceinline__ void umma_pool(uint32_t tmem_d, uint32_t tile_smem, uint32_t ind_smem, bool accumulate) {
 #pragma unroll
     for (int ks = 0; ks < 8; ++ks) {                     // 16 tokens per step
         const uint32_t a_addr = tile_smem + ks * 2048;
         const uint64_t da = uint64_t((a_addr >> 4) & 0x3fffu) | (uint64_t(kOpHalfBytes >> 4) << 16) |
                             (uint64_t(1024 >> 4) << 32) | (uint64_t(1) << 46) | (uint64_t(2) << 61);
         const uint64_t db = umma_desc_sw128(ind_smem + (ks >> 2) * (kIndBytes / 2) + (ks & 3) * 32);
-        umma_bf16(tmem_d, da, db, kIdescPool, ks ? 1u : 0u);
+        umma_bf16(tmem_d, da, db, kIdescPool, (accumulate || ks) ? 1u : 0u);
     }
 }
 // 16 consecutive fp32 columns of this thread's tensor-memory lane.
@@ -252,7 +253,8 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_consta
         for (int b = 0; b < kAccBufs; ++b) mbar_init(&ctl->tempty[b], 4);
         for (int g = 0; g < 4; ++g)
             for (int j = 0; j < 4; ++j) mbar_init(&ctl->tfull[g][j], 1);
-        for (int i = 0; i < kIndRing; ++i) { mbar_init(&ctl->ifull[i], kPoolWarps); mbar_init(&ctl->pfull[i], 1); }
+        for (int i = 0; i < kIndRing; ++i) { mbar_init(&ctl->ifull[i], kPoolWarps); mbar_init(&ctl->iempty[i], 1); }
+        for (int i = 0; i < 2; ++i) mbar_init(&ctl->pfull[i], 1);
         ctl->abort_flag = 0;
         mbar_fence_init();
         tmap_prefetch(&mapK);
@@ -472,81 +474,70 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_consta
     } else if (kSweep == 2 && warp < 2 + 4 * kGroups + kPoolWarps) {
         // ------------------------------------------------------------------ per-sentence sums of the key rows
         // The sums are a product on the tensor cores: (tile^T: channel x token) x (indicator: token x sentence slot).
-        // Slot 0 of a tile's first matrix is a sentence that starts at or before the tile's first token; a tile that
-        // touches more than 16 sentences (empty ones count) gets further matrices.  Each of the four warps writes a
-        // quarter of the matrix and arrives; one thread of a fifth warp issues the product, and while it runs every warp
-        // adds the previous product (a thread owns one channel) to the sums in global memory.
-        // Every warp keeps, one entry per lane, a window of the slab's sentence offsets starting at entry `base`
-        // (entries past the table read as "never starts"), refilled from global memory when a tile needs entries
-        // beyond it: loads from shared memory wait several hundred cycles here (the tensor core streams its operands
-        // from it), so the per-tile work touches shared memory only to write the matrix.
+        // A run of consecutive tiles whose sentences all fall among the 16 sentences B .. B + 15 shares one accumulator
+        // (slot j = sentence B + j; the products of the run accumulate), so the sums are read out and added to global
+        // memory once per run, about every fifth tile.  Each of the four warps writes a quarter of a tile's matrix and
+        // arrives; one thread of a fifth warp issues the product; when a tile opens a new run the four warps read out the
+        // run before it (a thread owns one channel) while the new one is being multiplied.  A tile that touches more
+        // than 16 sentences (empty ones count) gets several matrices, each a run of its own.
+        // Every warp keeps, one entry per lane, the sentence offsets B .. B + 31 of the current run (entries past the
+        // table read as "never starts"), fetched from global memory when a run opens: loads from shared memory wait
+        // several hundred cycles here (the tensor core streams its operands from it), so the per-tile work touches
+        // shared memory only to write the matrix.
         constexpr int kNever = 0x7fffffff;
         const int gw = warp - (2 + 4 * kGroups);                // warp of the group: slots 4 gw .. 4 gw + 3 of a matrix
         const int gtid = tid - (2 + 4 * kGroups) * 32;
         const int quarter = warp & 3;                           // tensor-memory lanes this warp may read
         const int ch = quarter * 32 + lane;
         const uint32_t lane_addr = tmem_base + (uint32_t(quarter * 32) << 16) + kPoolCol;
-        int slab = slab0, S = 0, N = 0, ic = 0, first = 0, base = 0, w = kNever;
+        int slab = slab0, S = 0, N = 0, first = 0;
+        int ic = 0;                                             // indicator matrices written so far
+        int run = -1, B = 0, w = kNever;                        // current run: index, sentence of slot 0, offsets B + lane
+        uint32_t run_held = 0;                                  // its slots that hold tokens so far
+        int run_slab = 0;
         const int32_t* so = a.sent_off;
         bool ok = true, have = false;
-        // the product still to be drained: its accumulator, sentence of slot 0, slots that hold tokens
-        bool pend = false;
-        int p_slab = 0, p_first = 0;
-        uint32_t p_held = 0;
-        auto refill = [&](int b) { base = b; w = (b + lane <= S) ? so[b + lane] : kNever; };
-        auto drain = [&]() {
-            const int is = (ic - 1) & (kIndRing - 1);
-            ok = role_wait(&ctl->pfull[is], uint32_t((ic - 1) / kIndRing) & 1u, limit, &ctl->abort_flag, a.status);
-            ok = __all_sync(0xffffffffu, ok);
-            if (ok) {
-                tc_fence_after();
-                float v[kIndSlots];
-                tmem_ld16(lane_addr + uint32_t(is) * kIndSlots, v);
-                tc_fence_before();
-                float* dst = a.vsum + (size_t(p_slab) * a.max_sent + p_first) * kHeadDim + ch;
-#pragma unroll
-                for (int j = 0; j < kIndSlots; ++j)
-                    if (p_held & (1u << j)) atomicAdd(dst + size_t(j) * kHeadDim, v[j]);
+        // 32-way search for the last sentence that starts at or before token `tok`, one probe per lane
+        auto holder = [&](int tok) {
+            int lo = 0, len = S;
+            while (len > 32) {
+                const int stride = (len + 31) >> 5;
+                const int pidx = lo + lane * stride;
+                const bool le = pidx < lo + len && so[pidx] <= tok;
+                const int adv = max(__popc(__ballot_sync(0xffffffffu, le)) - 1, 0) * stride;
+                len = min(stride, len - adv);
+                lo += adv;
             }
-            pend = false;
+            const bool le = lane < len && so[lo + lane] <= tok;
+            return lo + max(__popc(__ballot_sync(0xffffffffu, le)) - 1, 0);
+        };
+        // read out run r (accumulator r & 1) and add it to the sums
+        auto drain = [&](int r, int r_slab, int r_B, uint32_t r_held) {
+            ok = role_wait(&ctl->pfull[r & 1], uint32_t(r >> 1) & 1u, limit, &ctl->abort_flag, a.status);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) return;
+            tc_fence_after();
+            float v[kIndSlots];
+            tmem_ld16(lane_addr + uint32_t(r & 1) * kIndSlots, v);
+            tc_fence_before();
+            float* dst = a.vsum + (size_t(r_slab) * a.max_sent + r_B) * kHeadDim + ch;
+#pragma unroll
+            for (int j = 0; j < kIndSlots; ++j)
+                if (r_held & (1u << j)) atomicAdd(dst + size_t(j) * kHeadDim, v[j]);
         };
         for (int tl = 0; tl < ntl && ok; ++tl) {
             const int t = t_begin + tl;
             const bool fresh = !have || pref[slab + 1] <= t;
-            int w0 = kNever;
             if (fresh) {
                 while (pref[slab + 1] <= t) ++slab;
                 have = true;
                 so = a.sent_off + size_t(slab) * (a.max_sent + 1);
-                w0 = lane <= a.max_sent ? so[lane] : kNever;        // issued together with the loads of the lengths
                 S = min(max(a.n_sent[slab], 0), a.max_sent);
                 N = live(slab);
             }
-            const int tok0 = (t - pref[slab]) * 128, valid = min(128, N - tok0);
+            const int tok0 = (t - pref[slab]) * 128, valid = min(128, N - tok0), tok_end = tok0 + valid;
             const int stage = tl % a.stages;
-            if (fresh) {
-                // the last sentence that starts at or before the first token: at the head of a slab it is among the first
-                // entries (already loaded) unless the slab opens with 32 empty sentences
-                base = 0;
-                w = lane <= S ? w0 : kNever;
-                const int n_le = __popc(__ballot_sync(0xffffffffu, lane < S && w <= tok0));
-                first = max(n_le - 1, 0);
-            }
-            if (fresh && (tok0 > 0 || first >= 31)) {
-                // elsewhere: a 32-way search, one probe per lane
-                int lo = 0, len = S;
-                while (len > 32) {
-                    const int stride = (len + 31) >> 5;
-                    const int pidx = lo + lane * stride;
-                    const bool le = pidx < lo + len && so[pidx] <= tok0;
-                    const int adv = max(__popc(__ballot_sync(0xffffffffu, le)) - 1, 0) * stride;
-                    len = min(stride, len - adv);
-                    lo += adv;
-                }
-                const bool le = lane < len && so[lo + lane] <= tok0;
-                first = lo + max(__popc(__ballot_sync(0xffffffffu, le)) - 1, 0);
-                refill(first);
-            }
+            if (fresh) first = tok0 > 0 ? holder(tok0) : 0;     // (a slab that opens with empty sentences: they get slots)
             // every warp follows every tile's arrival (in order, so it sees each phase of the stage's barrier)
             ok = role_wait(&ctl->full[stage], uint32_t(tl / a.stages) & 1u, limit, &ctl->abort_flag, a.status);
             ok = __all_sync(0xffffffffu, ok);
@@ -560,44 +551,60 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_consta
                     *reinterpret_cast<uint4*>(tile + kOpHalfBytes + u * 16) = make_uint4(0u, 0u, 0u, 0u);
                 }
             }
+            int cur = first;                                    // first sentence of the tile not yet in a matrix
             int more = 0;
             do {
-                const int is = ic & (kIndRing - 1);
-                if (first < base || first + kIndSlots > base + 31) refill(first);
-                const int d = first - base;                         // window position of slot 0's sentence
-                // tile-relative start of every window entry, clamped to the tile; slot j holds [cl(d + j), cl(d + j + 1))
-                const int cl = min(max(min(w, tok0 + valid) - tok0, 0), valid);
+                // can the tile (from sentence cur on) join the open run?  its last sentence must be below B + 16
+                bool join = false;
+                if (run >= 0 && !fresh && cur >= B && cur - B < kIndSlots) {
+                    const int touching = __popc(__ballot_sync(0xffffffffu, lane > cur - B && B + lane < S && w < tok_end));
+                    join = cur + touching - B < kIndSlots;
+                }
+                const int r_prev = run, p_slab = run_slab, p_B = B;
+                const uint32_t p_held = run_held;
+                if (!join) {                                    // open a run at sentence cur
+                    ++run; B = cur; run_slab = slab; run_held = 0;
+                    w = (B + lane <= S) ? so[B + lane] : kNever;
+                }
+                // tile-relative start of the sentences B + lane, clamped to the tile; slot j holds [cl(j), cl(j + 1))
+                const int cl = min(max(min(w, tok_end) - tok0, 0), valid);
                 const int cl_next = __shfl_down_sync(0xffffffffu, cl, 1);
-                const uint32_t holds = __ballot_sync(0xffffffffu, base + lane < S && lane < 31 && cl_next > cl);
-                const uint32_t held = (holds >> d) & 0xffffu;       // bit j: slot j holds tokens
-                const int s_next = __shfl_sync(0xffffffffu, w, d + kIndSlots);   // start of the sentence after slot 15
-                more = (first + kIndSlots < S && s_next < tok0 + valid) ? 1 : 0;
-                // sentences after slot 0 that start at or before the next tile's first token: the last of them is a
-                // valid slot 0 there
-                const bool in_next = lane > d && lane <= d + kIndSlots && base + lane < S && w <= tok0 + 128;
-                const int step = __popc(__ballot_sync(0xffffffffu, in_next));
+                const uint32_t held = __ballot_sync(0xffffffffu, lane < kIndSlots && B + lane < S && cl_next > cl);
+                const int s_next = __shfl_sync(0xffffffffu, w, kIndSlots);           // start of the sentence after slot 15
+                more = (B + kIndSlots < S && s_next < tok_end) ? 1 : 0;
+                const int is = ic & (kIndRing - 1);
+                if (ic >= kIndRing) {                           // the product that read this buffer last has completed
+                    ok = role_wait(&ctl->iempty[is], uint32_t(ic / kIndRing - 1) & 1u, limit, &ctl->abort_flag, a.status);
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                }
                 {
-                    const int j = 4 * gw + (lane >> 3);             // this thread's slot row and its two pieces
-                    const int lo = __shfl_sync(0xffffffffu, cl, d + j), hi = __shfl_sync(0xffffffffu, cl, d + j + 1);
+                    const int j = 4 * gw + (lane >> 3);         // this thread's slot row and its two pieces
+                    const int lo = __shfl_sync(0xffffffffu, cl, j), hi = __shfl_sync(0xffffffffu, cl, j + 1);
                     const bool is_sent = (held >> j) & 1u;
                     indicator_piece(indb + size_t(is) * kIndBytes, j, (lane & 7) * 2, is_sent ? lo : 0, is_sent ? hi : 0);
                     indicator_piece(indb + size_t(is) * kIndBytes, j, (lane & 7) * 2 + 1, is_sent ? lo : 0, is_sent ? hi : 0);
                 }
-                fence_proxy_async_smem();                           // the matrix (and cleared rows) are read by the tensor core
-                tc_fence_before();                                  // and this warp's reads of the accumulator came first
+                fence_proxy_async_smem();                       // the matrix (and cleared rows) are read by the tensor core
+                tc_fence_before();                              // and this warp's reads of the accumulators came first
                 __syncwarp();
                 if (lane == 0) {
-                    if (gw == 0) ctl->ind_more[is] = more;
+                    if (gw == 0) ctl->ind_flags[is] = more | (join ? 2 : 0) | ((!join && r_prev >= 0) ? 4 : 0);
                     mbar_arrive(&ctl->ifull[is]);
                 }
-                if (pend) drain();                                  // the previous product, while this one runs
-                if (!ok) break;
-                pend = true; p_slab = slab; p_first = first; p_held = held;
+                run_held |= held;
                 ++ic;
-                first = more ? first + kIndSlots : first + step;
+                if (!join && r_prev >= 0) {                     // the run before, while the new one is being multiplied
+                    drain(r_prev, p_slab, p_B, p_held);
+                    if (!ok) break;
+                }
+                cur = B + kIndSlots;
             } while (more);
+            // the next tile starts in the last sentence of the run's window that starts at or before its first token
+            const int n_le = __popc(__ballot_sync(0xffffffffu, B + lane < S && w <= tok0 + 128));
+            first = (n_le == 32 && B + 32 < S) ? holder(tok0 + 128) : B + max(n_le - 1, 0);
         }
-        if (pend && ok) drain();
+        if (ok && run >= 0) drain(run, run_slab, B, run_held);  // the issuer closes the last run when its tiles are done
     } else if (kSweep == 2) {
         // ------------------------------------------------------------------ issuer of the pooling products
         // (its own thread: an issue blocks for the length of the product, and every look at shared memory costs the
@@ -605,23 +612,26 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_consta
         if (lane == 0 && ntl > 0) {
             const uint32_t indb_u32 = smem_u32(indb);
             bool ok = true;
-            int pc = 0;
+            int pc = 0, run = -1;
             for (int tl = 0; tl < ntl && ok; ++tl) {
                 const int stage = tl % a.stages;
-                int more = 0;
+                int flags = 0;
                 do {
                     const int is = pc & (kIndRing - 1);
                     ok = role_wait(&ctl->ifull[is], uint32_t(pc / kIndRing) & 1u, limit, &ctl->abort_flag, a.status);
                     if (!ok) break;
-                    more = *reinterpret_cast<volatile int*>(&ctl->ind_more[is]);
+                    flags = *reinterpret_cast<volatile int*>(&ctl->ind_flags[is]);       // 1: more, 2: joins the run, 4: closes one
                     tc_fence_after();
-                    umma_pool(tmem_base + kPoolCol + uint32_t(is) * kIndSlots, smem_u32(tiles + size_t(stage) * kOpBytes),
-                              indb_u32 + uint32_t(is) * kIndBytes);
-                    umma_commit(&ctl->pfull[is]);
+                    if (flags & 4) umma_commit(&ctl->pfull[run & 1]);                    // everything of the run before is issued
+                    if (!(flags & 2)) ++run;
+                    umma_pool(tmem_base + kPoolCol + uint32_t(run & 1) * kIndSlots, smem_u32(tiles + size_t(stage) * kOpBytes),
+                              indb_u32 + uint32_t(is) * kIndBytes, (flags & 2) != 0);
+                    umma_commit(&ctl->iempty[is]);
                     ++pc;
-                } while (more);
+                } while (flags & 1);
                 if (ok) umma_commit(&ctl->empty[stage]);
             }
+            if (ok && run >= 0) umma_commit(&ctl->pfull[run & 1]);
         }
     }
     tc_fence_before();
