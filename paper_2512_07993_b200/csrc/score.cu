@@ -16,10 +16,11 @@
 //
 // Both sweeps are persistent, warp-specialised kernels, one CTA per SM: a TMA warp streams
 // 128-token key tiles (and the group's query block) into shared memory, one thread issues
-// tcgen05.mma into a ring of four tensor-memory accumulators, several warpgroups of epilogue warps
-// take the tiles round-robin, and (sweep 2) one more warpgroup builds the 0/1 matrices of the pooling product,
-// issues it and drains the pooled sums.  Work is the list of
-// 128-token tiles over all slabs cut into equal contiguous ranges, so ragged slabs balance.
+// tcgen05.mma into a ring of tensor-memory accumulators (four in sweep 1, three in sweep 2), several
+// warpgroups of epilogue warps take the tiles round-robin, and (sweep 2) one more warpgroup writes the 0/1
+// matrices of the pooling product and reads out the pooled sums while one thread of a further warp issues
+// that product.  Work is the list of 128-token tiles over all slabs cut into equal contiguous ranges, so
+// ragged slabs balance.
 //
 // Query rows of a group are staged as blocks of WB = floor(128/n) window positions x n heads
 // (row q*WB + w of a block), so that the n heads of a window position sit at a fixed column
