@@ -434,8 +434,9 @@ def main():
     line = {"metric": METRIC, "value": replica_value(evict_us, world), "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": step_ms, "higher_is_better": False, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16 storage, f32 arithmetic", "data": "synthetic",
-            "config": workload_config(cfg, args.config, int(kv0.sum() // cfg.n_kv_heads // NL),
-                                      int(kv1.sum() // cfg.n_kv_heads // NL), NL, world),
+            # token counts of the first layer (the layer the reference arm runs), so that both arms name the same numbers
+            "config": workload_config(cfg, args.config, int(kv0[0].sum() // cfg.n_kv_heads),
+                                      int(kv1[0].sum() // cfg.n_kv_heads), NL, world),
             "us": us, "decode_attn_us": dec_us_max, "decode_attn_gbs": bytes_alg["decode_attn"] / (dec_us_max * 1e-6) / 1e9,
             "roofline": dict(roof[dominant], kernel=dominant), "roofline_by_step": roof,
             "gpu_launches": sum(LAUNCHES_PER_STEP.values()) * NL * args.steps, "clocks": clk}
