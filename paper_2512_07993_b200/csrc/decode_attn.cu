@@ -80,9 +80,10 @@ struct DecSmem {
 
 __device__ __forceinline__ void consumer_bar() { asm volatile("bar.sync 1, %0;" ::"n"(kConsWarps * 32) : "memory"); }
 
-// One consumer warp, 8 rows [row_base, row_base+8) of a tile, heads hg*4 .. hg*4+3.
-template <bool kGuard>
-__device__ __forceinline__ void tile_rows(const uint8_t* Ks, const uint8_t* Vs, int row_base, int rows, int lane,
+// One consumer warp, 8 rows [row_base, row_base+8) of a tile, the kH (1..4) heads of the warp's head group: the
+// multiply-adds are done for those heads only, the reduction always runs over four head slots.
+template <bool kGuard, int kH>
+__device__ __forceinline__ void tile_rows_h(const uint8_t* Ks, const uint8_t* Vs, int row_base, int rows, int lane,
                                           const float2 (&q2)[4][4], float2 (&acc)[4][4], float& m_run,
                                           float& l_run) {
     const int half = lane >> 4, l16 = lane & 15;
@@ -96,11 +97,15 @@ __device__ __forceinline__ void tile_rows(const uint8_t* Ks, const uint8_t* Vs, 
                      k3 = bf16x2_to_f2(kk.w);
 #pragma unroll
         for (int h = 0; h < 4; ++h) {
-            float2 a = __fmul2_rn(q2[h][0], k0);
-            a = __ffma2_rn(q2[h][1], k1, a);
-            a = __ffma2_rn(q2[h][2], k2, a);
-            a = __ffma2_rn(q2[h][3], k3, a);
-            part[i * 4 + h] = a.x + a.y;
+            if (h < kH) {
+                float2 a = __fmul2_rn(q2[h][0], k0);
+                a = __ffma2_rn(q2[h][1], k1, a);
+                a = __ffma2_rn(q2[h][2], k2, a);
+                a = __ffma2_rn(q2[h][3], k3, a);
+                part[i * 4 + h] = a.x + a.y;
+            } else {
+                part[i * 4 + h] = 0.f;
+            }
         }
     }
     // butterfly over the 16 lanes of a half-warp: lane l16 ends with the full sum of part[l16]
@@ -139,7 +144,7 @@ __device__ __forceinline__ void tile_rows(const uint8_t* Ks, const uint8_t* Vs, 
         const float sc = ex2(m_run - m_new);             // first block: 2^(-inf) = 0
         l_run *= sc;
 #pragma unroll
-        for (int h = 0; h < 4; ++h) {
+        for (int h = 0; h < kH; ++h) {
             const float sh = __shfl_sync(0xffffffffu, sc, h);
             const float2 s2 = make_float2(sh, sh);
 #pragma unroll
@@ -158,7 +163,7 @@ __device__ __forceinline__ void tile_rows(const uint8_t* Ks, const uint8_t* Vs, 
         const float2 v0 = bf16x2_to_f2(vv.x), v1 = bf16x2_to_f2(vv.y), v2 = bf16x2_to_f2(vv.z),
                      v3 = bf16x2_to_f2(vv.w);
 #pragma unroll
-        for (int h = 0; h < 4; ++h) {
+        for (int h = 0; h < kH; ++h) {
             const float ph = __shfl_sync(0xffffffffu, p, (lane & 16) | (i * 4 + h));
             const float2 pp = make_float2(ph, ph);
             acc[h][0] = __ffma2_rn(pp, v0, acc[h][0]);
@@ -169,9 +174,27 @@ __device__ __forceinline__ void tile_rows(const uint8_t* Ks, const uint8_t* Vs, 
     }
 }
 
+template <bool kGuard, bool kExact>
+__device__ __forceinline__ void tile_rows(int heads, const uint8_t* Ks, const uint8_t* Vs, int row_base, int rows, int lane,
+                                          const float2 (&q2)[4][4], float2 (&acc)[4][4], float& m_run, float& l_run) {
+    if (!kExact) {
+        tile_rows_h<kGuard, 4>(Ks, Vs, row_base, rows, lane, q2, acc, m_run, l_run);
+        return;
+    }
+    switch (heads) {                                         // the same for every thread of a warp
+        case 4: tile_rows_h<kGuard, 4>(Ks, Vs, row_base, rows, lane, q2, acc, m_run, l_run); break;
+        case 3: tile_rows_h<kGuard, 3>(Ks, Vs, row_base, rows, lane, q2, acc, m_run, l_run); break;
+        case 2: tile_rows_h<kGuard, 2>(Ks, Vs, row_base, rows, lane, q2, acc, m_run, l_run); break;
+        default: tile_rows_h<kGuard, 1>(Ks, Vs, row_base, rows, lane, q2, acc, m_run, l_run); break;
+    }
+}
+
+// kExact: head groups of equal size with the multiply-adds of a warp limited to its group's heads (for group sizes
+// that are not a multiple of four; a separate instance, so that the common four-heads-per-group kernel carries one
+// copy of the row code, not four).
 // kStep: the launch also performs the per-step bookkeeping described at StepArgs (a separate instance, so that
 // plain decode attention carries none of it).
-template <bool kStep>
+template <bool kStep, bool kExact>
 __global__ void __launch_bounds__(kDecThreads, kCtasPerSm)
 decode_attn_kernel(int batch, int Hq, int Hk, int n_slabs, const int64_t* slab_off, const int32_t* cap,
                    const __nv_bfloat16* q, const uint8_t* K, const uint8_t* V, const int32_t* kv_len,
@@ -197,7 +220,8 @@ decode_attn_kernel(int batch, int Hq, int Hk, int n_slabs, const int64_t* slab_o
     // rows streamed through the tile ring; with the fused step the row being appended is folded in separately
     auto live = [&](int s) { return old_len(s); };
     const int n = Hq / Hk;                     // heads per group
-    const int NG = (n + 3) / 4;                // head groups of 4 (1 or 2)
+    const int NG = (n + 3) / 4;                // head groups (1 or 2) of H0 heads each, the last one possibly smaller:
+    const int H0 = kExact ? (n + NG - 1) / NG : 4;   // exact: 5 heads are 3 + 2, not 4 + 1, and no warp multiplies for absent heads
     const int G = gridDim.x, cta = blockIdx.x;
 
     if (tid == 0) {
@@ -239,6 +263,7 @@ decode_attn_kernel(int batch, int Hq, int Hk, int n_slabs, const int64_t* slab_o
 
     {
         const int hg = warp % NG;                       // head group of this warp
+        const int Hg = min(H0, n - hg * H0);            // its heads
         const int rb = warp / NG;                       // row block: rows [rb*NG*8, (rb+1)*NG*8) of each tile
         const int half = lane >> 4, l16 = lane & 15;
         const float qscale = 1.4426950408889634f * rsqrtf(float(kHeadDim));
@@ -361,9 +386,9 @@ decode_attn_kernel(int batch, int Hq, int Hk, int n_slabs, const int64_t* slab_o
             }
 #pragma unroll
             for (int hh = 0; hh < 4; ++hh) {
-                const int hl = hg * 4 + hh;
+                const int hl = hg * H0 + hh;
                 uint4 qq = make_uint4(0u, 0u, 0u, 0u);
-                if (hl < n)
+                if (hh < Hg)
                     qq = reinterpret_cast<const uint4*>(q + (size_t(b) * Hq + size_t(h) * n + hl) * kHeadDim)[l16];
                 const float2 s2 = make_float2(qscale, qscale);
                 q2[hh][0] = __fmul2_rn(bf16x2_to_f2(qq.x), s2);
@@ -389,12 +414,12 @@ decode_attn_kernel(int batch, int Hq, int Hk, int n_slabs, const int64_t* slab_o
                     const uint8_t* Vs = Ks + kTileBytes;
                     if (rows_left >= kTileRows) {
                         for (int sub = 0; sub < NG; ++sub)
-                            tile_rows<false>(Ks, Vs, (rb * NG + sub) * 8, kTileRows, lane, q2, acc, m_run, l_run);
+                            tile_rows<false, kExact>(Hg, Ks, Vs, (rb * NG + sub) * 8, kTileRows, lane, q2, acc, m_run, l_run);
                     } else {
                         for (int sub = 0; sub < NG; ++sub) {
                             const int row_base = (rb * NG + sub) * 8;
                             if (row_base >= rows_left) break;
-                            tile_rows<true>(Ks, Vs, row_base, rows_left, lane, q2, acc, m_run, l_run);
+                            tile_rows<true, kExact>(Hg, Ks, Vs, row_base, rows_left, lane, q2, acc, m_run, l_run);
                         }
                     }
                     __syncwarp();
@@ -407,7 +432,7 @@ decode_attn_kernel(int batch, int Hq, int Hk, int n_slabs, const int64_t* slab_o
             if (own_tail && seg_append) {
                 consumer_bar();                            // the staged row is visible
                 if (warp < NG && !aborted)                 // one warp per head group folds the row into its running state
-                    tile_rows<true>(reinterpret_cast<const uint8_t*>(wpart), reinterpret_cast<const uint8_t*>(wpart) + 2048, 0, 1,
+                    tile_rows<true, kExact>(Hg, reinterpret_cast<const uint8_t*>(wpart), reinterpret_cast<const uint8_t*>(wpart) + 2048, 0, 1,
                                     lane, q2, acc, m_run, l_run);
                 consumer_bar();                            // before the flush reuses the buffer
             }
@@ -448,7 +473,7 @@ decode_attn_kernel(int batch, int Hq, int Hk, int n_slabs, const int64_t* slab_o
             float* rec = dec_part + size_t(cta + slab) * n * kPartStride;
             for (int idx = tid; idx < n * kHeadDim; idx += kConsWarps * 32) {
                 const int hl = idx / kHeadDim, c = idx % kHeadDim;
-                const int g2 = hl / 4, hh = hl % 4;
+                const int g2 = hl / H0, hh = hl % H0;
                 float M = -INFINITY;
                 for (int w = g2; w < kConsWarps; w += NG) M = fmaxf(M, wpart[(w * 4 + hh) * kWpStride + 128]);
                 float L = 0.f, A = 0.f;
@@ -563,7 +588,9 @@ static int decode_impl(const skipkv_shape* shape, const void* q, const void* K, 
         return SKIPKV_ERR_UNSUPPORTED;
     }
     // set on every call: the attribute belongs to the current device's context, which a cached value would not track
-    auto kern = step.k_new ? decode_attn_kernel<true> : decode_attn_kernel<false>;
+    const bool exact = (shape->n_q_heads / shape->n_kv_heads) % 4 != 0;
+    auto kern = step.k_new ? (exact ? decode_attn_kernel<true, true> : decode_attn_kernel<true, false>)
+                           : (exact ? decode_attn_kernel<false, true> : decode_attn_kernel<false, false>);
     SKIPKV_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
     int grid = num_sms() * kCtasPerSm;
     if (grid > L.dec_max_ctas) grid = L.dec_max_ctas;
@@ -713,7 +740,7 @@ extern "C" int skipkv_decode_attn_static(const skipkv_shape* shape, const void* 
                         size_t(slabs + 1) * 4;
     unsigned char* base = nullptr;
     if (int rc = static_setup(dev, &base)) return rc;
-    SKIPKV_CUDA(cudaFuncSetAttribute(decode_attn_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
+    SKIPKV_CUDA(cudaFuncSetAttribute(decode_attn_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     // The array keeps whatever the previous call left: the status word and the arrival counters
     // must start at zero (the partial records are fully written before they are read).
@@ -721,7 +748,7 @@ extern "C" int skipkv_decode_attn_static(const skipkv_shape* shape, const void* 
     int grid = num_sms() * kCtasPerSm;
     if (grid > kStaticMaxCtas) grid = kStaticMaxCtas;
     uint32_t* status_word = status ? status : reinterpret_cast<uint32_t*>(base);
-    decode_attn_kernel<false><<<grid, kDecThreads, smem, st>>>(
+    decode_attn_kernel<false, false><<<grid, kDecThreads, smem, st>>>(
         shape->batch, shape->n_q_heads, shape->n_kv_heads, slabs, shape->slab_off, shape->cap,
         static_cast<const __nv_bfloat16*>(q), static_cast<const uint8_t*>(K), static_cast<const uint8_t*>(V), kv_len,
         static_cast<__nv_bfloat16*>(out), status_word, reinterpret_cast<uint32_t*>(base + kStaticCntOff),
