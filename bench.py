@@ -291,6 +291,56 @@ def time_extras(cfg, B, flush, clean, peaks, reps=10):
     D.status()
     del D
     torch.cuda.empty_cache()
+    # the decode loop itself (Algorithm 2): fused steps over a few layers, one sentence opened every 16 tokens, an eviction
+    # pass (score, select, compact on every layer) every 128 steps; event times, the host loop's gaps included
+    n_layers, steps, interval = 4, 256, 128
+    cfgl = W.config(4, ctx_lo=2048, ctx_hi=2048, batch=cfg.batch)
+    Ds = []
+    for l in range(n_layers):
+        Ll = W.make_layer(cfgl, layer=l)
+        ms = int(Ll["max_sent"]) + steps                    # room for the sentences the loop opens
+        for key in ("sent_off", "sent_id"):
+            old = Ll[key]
+            new = np.zeros(old.shape[:2] + (ms + (1 if key == "sent_off" else 0),), np.int32)
+            new[..., :old.shape[2]] = old
+            new[..., old.shape[2]:] = old[..., -1:] if key == "sent_off" else -1
+            Ll[key] = new
+        Ll["max_sent"] = ms
+        Ds.append(B.DeviceLayer(Ll))
+    other = [torch.zeros_like(D.kv_len) for D in Ds]
+    k_new = torch.randn(cfgl.batch, cfgl.n_kv_heads, 128, device=dev).bfloat16(); v_new = torch.randn_like(k_new)
+    opens = [torch.full((cfgl.batch,), 1 if t % 16 == 0 else 0, dtype=torch.uint8, device=dev) for t in range(2)]
+    gen = torch.zeros(cfgl.batch, dtype=torch.int32, device=dev)
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    t_step, t_evict, n_evict = 0.0, 0.0, 0
+    marks = []
+    e_prev = ev(); e_prev.record()
+    for t in range(steps):
+        for l, D in enumerate(Ds):
+            B.skipkv_decode_step(D.shape, D.q, k_new, v_new, D.K, D.V, D.kv_len, other[l], D.sent_off, D.sent_id, D.n_sent,
+                                 opens[1 if t % 16 else 0], gen, D.q_win, t % cfgl.window, D.out, D.hidden, D.steer_vec,
+                                 D.alpha, D.flag, D.ws)
+            D.kv_len, other[l] = other[l], D.kv_len
+        if (t + 1) % interval == 0:
+            e0 = ev(); e0.record()
+            for D in Ds:
+                D.score(); D.select(); D.compact()
+            e1 = ev(); e1.record()
+            marks.append((e_prev, e0, e1))
+            e_prev = e1
+    e_end = ev(); e_end.record()
+    torch.cuda.synchronize()
+    for a0, b0, c0 in marks:
+        t_step += a0.elapsed_time(b0); t_evict += b0.elapsed_time(c0); n_evict += 1
+    t_step += e_prev.elapsed_time(e_end)
+    for D in Ds:
+        D.status()
+    out["decode_loop"] = {"layers": n_layers, "steps": steps, "evictions": n_evict, "rows_per_slab": "2048 .. 2176",
+                          "us_per_layer_step": t_step * 1e3 / (steps * n_layers),
+                          "us_per_layer_eviction": t_evict * 1e3 / max(n_evict * n_layers, 1),
+                          "note": "CUDA events around a Python loop of C-ABI calls: launch gaps of the host loop included"}
+    del Ds, other
+    torch.cuda.empty_cache()
     # token-level redundancy at the steady-state length of a budgeted cache: budget + 128 rows per slab
     n_tok = cfg.budget + 128
     cfg_ss = W.config(0, batch=cfg.batch, n_q_heads=cfg.n_q_heads, n_kv_heads=cfg.n_kv_heads, window=cfg.window,

@@ -66,6 +66,7 @@ struct SweepCtl {                       // barriers and small shared state, afte
     // the pooling warps
     uint64_t ifull[kIndRing], iempty[kIndRing];
     uint64_t pfull[2];                  // the last product of a run of tiles into accumulator i has completed
+    uint64_t issued_done[2];            // after a failed wait: every product of the MMA thread (0) / the pooling issuer (1) has retired
     int ind_flags[kIndRing];            // 1: the tile has another matrix after this one, 2: joins the open run, 4: closes a run
     uint32_t wsum[32];
     alignas(16) float neg_lse[kSw2Groups][kMaxRB * 128];   // sweep 2: one copy per epilogue warpgroup (read as float4)
@@ -255,7 +256,7 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_consta
         for (int g = 0; g < 4; ++g)
             for (int j = 0; j < 4; ++j) mbar_init(&ctl->tfull[g][j], 1);
         for (int i = 0; i < kIndRing; ++i) { mbar_init(&ctl->ifull[i], kPoolWarps); mbar_init(&ctl->iempty[i], 1); }
-        for (int i = 0; i < 2; ++i) mbar_init(&ctl->pfull[i], 1);
+        for (int i = 0; i < 2; ++i) { mbar_init(&ctl->pfull[i], 1); mbar_init(&ctl->issued_done[i], 1); }
         ctl->abort_flag = 0;
         mbar_fence_init();
         tmap_prefetch(&mapK);
@@ -371,6 +372,11 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_consta
                 if (t + 1 == t_end || slab_end <= t + 1) umma_commit(&ctl->qempty);
                 umma_commit(&ctl->empty[stage]);
                 if (++stage == a.stages) { stage = 0; ++lap; }
+            }
+            if (!ok) {
+                // nobody will wait for the products still in flight: let them retire before the tensor memory is released
+                umma_commit(&ctl->issued_done[0]);
+                mbar_wait(&ctl->issued_done[0], 0u, 1u << 18);
             }
         }
     } else if (warp < 2 + 4 * kGroups) {
@@ -633,6 +639,10 @@ score_sweep_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_consta
                 if (ok) umma_commit(&ctl->empty[stage]);
             }
             if (ok && run >= 0) umma_commit(&ctl->pfull[run & 1]);
+            if (!ok) {
+                umma_commit(&ctl->issued_done[1]);
+                mbar_wait(&ctl->issued_done[1], 0u, 1u << 18);
+            }
         }
     }
     tc_fence_before();
