@@ -152,6 +152,28 @@ __device__ __forceinline__ float imp_fold(uint32_t taddr, const float* neg_lse, 
         }
         return t0 + t1;
     }
+    if constexpr (kN > 4) {
+        // WB <= 25 window positions per head: one load of 32 columns per head, starting at the head's first column
+        // (the columns read past its last position are not used), in a rolled loop like the four-head case
+        float best[WB];
+#pragma unroll
+        for (int w = 0; w < WB; ++w) best[w] = -INFINITY;
+#pragma unroll 1
+        for (int q = 0; q < kN; ++q) {
+            float v[32];
+            tmem_ld32(taddr + q * WB, v);
+            const float* nl = neg_lse + q * WB;
+#pragma unroll
+            for (int w = 0; w < WB; ++w) best[w] = fmaxf(best[w], fmaf(v[w], scale, nl[w]));
+        }
+        float t0 = 0.f, t1 = 0.f;
+#pragma unroll
+        for (int w = 0; w < WB; w += 2) {
+            t0 += (w < wvalid) ? ex2f(best[w]) : 0.f;
+            if (w + 1 < WB) t1 += (w + 1 < wvalid) ? ex2f(best[w + 1]) : 0.f;
+        }
+        return t0 + t1;
+    }
     float best[WB];
     float total = 0.f;
 #pragma unroll
